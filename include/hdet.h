@@ -1,0 +1,236 @@
+/*
+ * hdet.h -- C ABI of libhdet: the per-step hot path of Hyperparameter-Divergent
+ * Ensemble Training (HDET, arXiv 2604.24708) with the N replicas stacked on one GPU.
+ *
+ * One handle drives Algorithm 1's loop body for a list of parameter tensors:
+ *
+ *   hdet_create        validate the tensor list, build the device work table
+ *   hdet_set_schedule  base schedule (Algorithm 1, Require) and controller constants
+ *   hdet_step          spread (Eq. 1) x base rate -> fused fan-out update (Eq. 2 /
+ *                      Adam, Section 4.1); on the last update of a round the converge
+ *                      mean (Eq. 3) is formed in the same kernel
+ *   hdet_converge      stand-alone converge (Eq. 3)
+ *   hdet_autolr_update controller (Eq. 4 - Eq. 9) after a converge
+ *   hdet_get_state / hdet_set_state   scalars for logging and resume
+ *   hdet_destroy
+ *
+ * Conventions
+ *   - Every tensor pointer is a DEVICE pointer owned by the caller; it must stay
+ *     valid until hdet_destroy.  Scalar arrays (losses, max_lr, ...) are HOST pointers
+ *     read during the call only.
+ *   - Layout: replica r of a tensor starts at base + r * stride (strides in elements).
+ *     Parameters and Adam moments are fp32.  Gradients are fp32 or bf16.
+ *   - All kernels are launched on the caller's stream (a cudaStream_t passed as
+ *     void*; NULL = the legacy default stream) and the calls return without
+ *     synchronising unless stated otherwise.  Launches of one handle must be ordered
+ *     on the device by the caller (same stream, or events).
+ *   - No function throws or aborts; each returns an hdet_status.  hdet_last_error
+ *     gives a text for the last failure on a handle.
+ *   - The library owns only its work table, a status word on the device and the host
+ *     controller state.  hdet_step / hdet_converge / hdet_autolr_update allocate nothing.
+ *   - There is no CPU fallback: a handle with tensors needs a CUDA device.  A handle
+ *     created with n_tensors == 0 touches no device and runs only the scalar part
+ *     (schedule, spread, controller), which is what host-side tests use.
+ */
+#ifndef HDET_H_
+#define HDET_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define HDET_API __attribute__((visibility("default")))
+#else
+#define HDET_API
+#endif
+
+#define HDET_MAX_REPLICAS 32
+#define HDET_MAX_GROUPS 8
+
+typedef enum {
+  HDET_OK = 0,
+  HDET_ERR_INVALID_ARG = 1, /* NULL pointer, value out of range                          */
+  HDET_ERR_STATE = 2,       /* call out of order (no schedule set, no round just ended)  */
+  HDET_ERR_ALIGN = 3,       /* a pointer is not aligned to its element type              */
+  HDET_ERR_UNSUPPORTED = 4, /* a valid request this build does not implement             */
+  HDET_ERR_CUDA = 5,        /* a CUDA runtime call failed; see hdet_last_error           */
+  HDET_ERR_NONFINITE = 6    /* a kernel produced a non-finite parameter (sticky)         */
+} hdet_status;
+
+enum { HDET_OPT_SGD = 0, HDET_OPT_ADAMW = 1 };
+enum { HDET_DTYPE_F32 = 0, HDET_DTYPE_BF16 = 1 };
+enum { HDET_SCHED_CONSTANT = 0, HDET_SCHED_ONECYCLE_COS = 1, HDET_SCHED_ONECYCLE_LINEAR = 2 };
+
+typedef struct hdet_ctx* hdet_handle;
+
+/* One parameter tensor with its N replicas.  Device pointers, caller-owned. */
+typedef struct {
+  void* param;          /* fp32 [N] x numel, replica stride param_stride                  */
+  void* grad;           /* fp32 or bf16 (hdet_config.grad_dtype), replica stride grad_stride */
+  void* exp_avg;        /* fp32 Adam first moment,  replica stride state_stride; NULL for SGD */
+  void* exp_avg_sq;     /* fp32 Adam second moment, replica stride state_stride; NULL for SGD */
+  int64_t numel;        /* elements per replica, > 0                                      */
+  int64_t param_stride; /* elements between replicas of param (>= numel when N > 1)       */
+  int64_t grad_stride;  /* elements between replicas of grad; 0 = one gradient shared by
+                           every replica (the all-reduced gradient of Eq. 2)              */
+  int64_t state_stride; /* elements between replicas of both moments                     */
+  int32_t group;        /* optimizer group, 0 .. n_groups-1                               */
+  int32_t reserved;     /* set to 0                                                       */
+} hdet_tensor;
+/* Alignment: pointers must be aligned to their element type (4 bytes fp32, 2 bytes
+ * bf16) or hdet_create returns HDET_ERR_ALIGN.  A tensor whose pointers are 16-byte
+ * aligned (gradients: 8 bytes for bf16, 16 for fp32) and whose strides are multiples of
+ * 4 elements takes the vectorised path; any other tensor is processed correctly by
+ * scalar loads. */
+
+typedef struct {
+  int32_t n_replicas;    /* N of Eq. 1, 1 .. HDET_MAX_REPLICAS                            */
+  int32_t n_groups;      /* optimizer parameter groups (Section 3.4), 1 .. HDET_MAX_GROUPS */
+  int32_t optimizer;     /* HDET_OPT_SGD (Eq. 2) or HDET_OPT_ADAMW (Section 4.1)          */
+  int32_t grad_dtype;    /* HDET_DTYPE_F32 or HDET_DTYPE_BF16                             */
+  double beta1, beta2, eps; /* Adam constants (ignored by SGD)                            */
+  double momentum;       /* SGD momentum; must be 0 (Eq. 2 has none)                      */
+  double alpha_lr;       /* spread ratio alpha of Eq. 1 for the learning rate, 0 <= a < 1 */
+  double alpha_wd;       /* spread ratio for the weight decay (Remark 1), 0 <= a < 1; 0 = none */
+  int64_t sync_interval; /* T of Section 3.3, >= 1                                        */
+  int32_t reshuffle;     /* 1: draw new permutations when the controller fires (Eq. 9)    */
+  int32_t fuse_converge; /* 1: the round's last update also forms the mean (one pass over
+                            the parameters); 0: update kernel then converge kernel        */
+  uint64_t seed;         /* seed of the permutation generator                             */
+  int32_t device;        /* CUDA device ordinal; ignored when n_tensors == 0              */
+  int32_t reserved;      /* set to 0                                                       */
+} hdet_config;
+
+/* Base schedule and controller constants (Algorithm 1, Require).  Host arrays with
+ * n_groups entries, copied during the call. */
+typedef struct {
+  int32_t kind;            /* HDET_SCHED_*                                                 */
+  int32_t autolr;          /* 1: run the auto-LR controller (Section 3.4)                  */
+  int64_t total_steps;     /* S                                                            */
+  const double* max_lr;    /* eta_max per group (the constant rate for HDET_SCHED_CONSTANT) */
+  const double* weight_decay; /* decoupled weight decay per group; NULL = all zero         */
+  double pct_start;        /* p: fraction of S spent rising; needs 1 < p*S < S             */
+  double div_factor;       /* initial rate = max_lr / div_factor                           */
+  double final_div_factor; /* final rate = initial rate / final_div_factor                 */
+  int64_t warmup_steps;    /* S_warm: the controller runs at syncs with t >= S_warm        */
+  double beta;             /* velocity momentum of Eq. 7                                   */
+  double sigma;            /* softmax temperature of Eq. 4, > 0                            */
+  double lambda;           /* velocity gain of Eq. 7                                       */
+  double f_div, f_final;   /* the two factors of Eq. 8, both > 0                           */
+} hdet_schedule;
+
+/* Scalar state for logging and resume.  Tables are [group][replica]. */
+typedef struct {
+  int64_t step;                       /* completed updates t                               */
+  int64_t n_acc;                      /* updates accumulated in loss_acc                   */
+  int32_t fired;                      /* the controller has taken over the base rate       */
+  int32_t round_ended;                /* the last hdet_step ended a round and
+                                         hdet_autolr_update has not run since             */
+  uint32_t device_status;             /* bit 0: a non-finite parameter was produced        */
+  int32_t reserved;
+  double base[HDET_MAX_GROUPS];       /* base rate used by the last update                 */
+  double ctrl_base[HDET_MAX_GROUPS];  /* eta_bar held by the controller (Eq. 7)            */
+  double velocity[HDET_MAX_GROUPS];   /* v of Eq. 7                                        */
+  double delta[HDET_MAX_GROUPS];      /* Delta of Eq. 6 at the last firing                 */
+  double lr[HDET_MAX_GROUPS][HDET_MAX_REPLICAS]; /* rates used by the last update          */
+  double wd[HDET_MAX_GROUPS][HDET_MAX_REPLICAS]; /* weight decays used by the last update  */
+  int32_t perm_lr[HDET_MAX_GROUPS][HDET_MAX_REPLICAS]; /* pi of Eq. 9, learning rate       */
+  int32_t perm_wd[HDET_MAX_GROUPS][HDET_MAX_REPLICAS]; /* pi of Eq. 9, weight decay        */
+  double weights[HDET_MAX_REPLICAS];   /* w of Eq. 4 at the last firing                    */
+  double loss_acc[HDET_MAX_REPLICAS];  /* running sum of losses in the current round       */
+  double loss_round[HDET_MAX_REPLICAS];/* mean loss per replica over the last full round   */
+  double gamma;                        /* decay of Eq. 8                                   */
+} hdet_state;
+
+/*
+ * hdet_create -- Algorithm 1, Init.  Checks cfg and the n_tensors descriptors, builds
+ * the device work table (one entry per tile of a tensor) and a device status word on
+ * cfg->device, and sets velocity 0, loss accumulator 0, identity permutations.
+ * tensors may be NULL only when n_tensors == 0.  On success *out receives the handle;
+ * on failure *out is NULL and nothing is left allocated.
+ * Errors: INVALID_ARG (NULL, N/G/T/alpha out of range, numel <= 0, group out of range,
+ * stride < numel with N > 1, missing moments for AdamW), ALIGN, UNSUPPORTED (momentum
+ * != 0), CUDA.
+ */
+HDET_API int hdet_create(const hdet_config* cfg, const hdet_tensor* tensors, int64_t n_tensors, hdet_handle* out);
+
+/*
+ * hdet_set_schedule -- stores the base schedule eta(t) named in Algorithm 1's Require
+ * list (one-cycle policy with cosine or linear annealing, or a constant) and the
+ * controller constants (beta, sigma, lambda of Eq. 4 / Eq. 7; f_div, f_final of Eq. 8;
+ * S_warm).  May be called again at any time; it does not reset the step count.
+ * Errors: INVALID_ARG (NULL, S < 1, max_lr NULL, p*S <= 1 or p >= 1 for a one-cycle
+ * kind, factors <= 0, sigma <= 0 with autolr, f_div or f_final <= 0).
+ */
+HDET_API int hdet_set_schedule(hdet_handle h, const hdet_schedule* sched);
+
+/*
+ * hdet_step -- one pass of Algorithm 1's loop body for update t = step + 1:
+ *   base_g   = controller's eta_bar_g once it has fired, else schedule_g(t - 1)
+ *   lr[g][r] = base_g * rho_{pi_g(r)}                 (Eq. 1, Section 3.2, Eq. 9)
+ *   wd[g][r] = wd_g * rho'_{pi'_g(r)}                 (Remark 1; rho' uses alpha_wd)
+ *   every replica of every tensor is updated in one kernel (Eq. 2, or Adam with
+ *   decoupled weight decay: theta *= 1 - lr*wd; m, v moving averages; theta -=
+ *   lr * (m/(1-beta1^t)) / (sqrt(v/(1-beta2^t)) + eps))
+ *   step_losses (HOST, N doubles, or NULL) are added to the round's accumulator
+ *   if t mod T == 0 the replicas are averaged (Eq. 3) -- inside the same kernel when
+ *   fuse_converge is set -- and *did_converge is set to 1 (else 0; may be NULL).
+ * Asynchronous on `stream`.  Scalars are computed in double on the host and handed to
+ * the kernel as fp32 launch parameters, so no host-to-device copy is issued.
+ * Errors: INVALID_ARG, STATE (no schedule), CUDA (launch failure).
+ */
+HDET_API int hdet_step(hdet_handle h, const double* step_losses, void* stream, int32_t* did_converge);
+
+/*
+ * hdet_converge -- Eq. 3 on its own: theta_r <- (1/N) sum_r' theta_r' for every tensor.
+ * Does not touch the step count, the moments or the loss accumulator.
+ * Errors: INVALID_ARG, CUDA.
+ */
+HDET_API int hdet_converge(hdet_handle h, void* stream);
+
+/*
+ * hdet_autolr_update -- the auto-LR branch of Algorithm 1, to be called after the
+ * hdet_step that set *did_converge.  With the round's mean losses L_r (round_losses,
+ * HOST, N doubles; NULL = the accumulated mean) it computes w (Eq. 4), per group
+ * Delta (Eq. 5 - 6) from the rates of the last update, the velocity and the new base
+ * eta_bar (Eq. 7, gamma from Eq. 8), and draws new permutations (Eq. 9) when
+ * reshuffle is set.  From then on hdet_step uses eta_bar as the group's base rate.
+ * It is a no-op returning HDET_OK when autolr is off or t < S_warm.  It runs on the
+ * host; `stream` is unused and may be NULL.
+ * Errors: INVALID_ARG, STATE (the last hdet_step did not end a round, or the update
+ * already ran for this round).
+ */
+HDET_API int hdet_autolr_update(hdet_handle h, const double* round_losses, void* stream);
+
+/*
+ * hdet_get_state -- copies the scalar state into *out.  Reads the device status word,
+ * which synchronises with the device (cudaMemcpy) when the handle has tensors.
+ * Returns HDET_ERR_NONFINITE (with *out filled) if a kernel flagged a non-finite value.
+ */
+HDET_API int hdet_get_state(hdet_handle h, hdet_state* out);
+
+/*
+ * hdet_set_state -- restores step, n_acc, fired, round_ended, ctrl_base, velocity, the
+ * permutations, loss_acc and loss_round from *in (resume); the other fields are
+ * recomputed.  Clears the device status word.
+ * Errors: INVALID_ARG (NULL, negative step, an array that is not a permutation).
+ */
+HDET_API int hdet_set_state(hdet_handle h, const hdet_state* in);
+
+/* hdet_destroy -- frees the work table and the handle.  NULL is accepted. */
+HDET_API int hdet_destroy(hdet_handle h);
+
+/* hdet_last_error -- text of the last failure on h (or of the last failed hdet_create
+ * when h is NULL).  The pointer stays valid until the next call on that handle. */
+HDET_API const char* hdet_last_error(hdet_handle h);
+
+/* hdet_kernel_launches -- number of kernels this handle has launched so far. */
+HDET_API int64_t hdet_kernel_launches(hdet_handle h);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HDET_H_ */

@@ -1,0 +1,70 @@
+"""Device memory layout helper: N replicas of a ragged tensor list packed into stacked arenas.
+
+Layout in HBM (one allocation per quantity, no per-tensor allocations):
+
+    param      fp32  [N][P_pad]     replica r of tensor k at  r * P_pad + offset_k
+    exp_avg    fp32  [N][P_pad]     (AdamW only)
+    exp_avg_sq fp32  [N][P_pad]     (AdamW only)
+    grad       fp32 or bf16 [N][P_pad]   (or [P_pad] when one gradient is shared)
+
+Every offset_k is a multiple of ``align_elems`` (8 by default: 32 bytes of fp32, 16 bytes of
+bf16), so every tensor takes the library's 128-bit path.  Only memory and descriptors are
+handled here; all arithmetic is in the CUDA library.
+"""
+from __future__ import annotations
+
+from typing import List, Sequence
+
+import torch
+
+from . import binding as B
+
+
+class StackedArena:
+    def __init__(self, numels: Sequence[int], groups: Sequence[int], n_replicas: int, optimizer: int,
+                 grad_dtype: int, device: str = "cuda:0", align_elems: int = 8, shared_grad: bool = False):
+        if not torch.cuda.is_available():
+            raise RuntimeError("StackedArena needs a CUDA device (there is no CPU path)")
+        self.numels = [int(x) for x in numels]
+        self.groups = [int(g) for g in groups]
+        self.n = int(n_replicas)
+        self.optimizer = optimizer
+        self.grad_dtype = grad_dtype
+        self.device = torch.device(device)
+        a = int(align_elems)
+        self.offsets: List[int] = []
+        cur = 0
+        for ne in self.numels:
+            self.offsets.append(cur)
+            cur += (ne + a - 1) // a * a
+        self.p_pad = cur
+        gd = torch.bfloat16 if grad_dtype == B.HDET_DTYPE_BF16 else torch.float32
+        self.param = torch.zeros((self.n, self.p_pad), dtype=torch.float32, device=self.device)
+        adam = optimizer == B.HDET_OPT_ADAMW
+        self.exp_avg = torch.zeros_like(self.param) if adam else None
+        self.exp_avg_sq = torch.zeros_like(self.param) if adam else None
+        self.shared_grad = bool(shared_grad)
+        gshape = (self.p_pad,) if shared_grad else (self.n, self.p_pad)
+        self.grad = torch.zeros(gshape, dtype=gd, device=self.device)
+
+    def descriptors(self) -> List[B.hdet_tensor]:
+        out = []
+        gsz = self.grad.element_size()
+        for off, ne, grp in zip(self.offsets, self.numels, self.groups):
+            t = B.hdet_tensor()
+            t.param = self.param.data_ptr() + 4 * off
+            t.grad = self.grad.data_ptr() + gsz * off
+            if self.exp_avg is not None:
+                t.exp_avg = self.exp_avg.data_ptr() + 4 * off
+                t.exp_avg_sq = self.exp_avg_sq.data_ptr() + 4 * off
+            t.numel = ne
+            t.param_stride = self.p_pad
+            t.grad_stride = 0 if self.shared_grad else self.p_pad
+            t.state_stride = self.p_pad
+            t.group = grp
+            out.append(t)
+        return out
+
+    def resident_bytes(self) -> int:
+        ts = [self.param, self.grad] + ([self.exp_avg, self.exp_avg_sq] if self.exp_avg is not None else [])
+        return sum(t.numel() * t.element_size() for t in ts)

@@ -1,0 +1,450 @@
+// C ABI of libhdet (see include/hdet.h): argument checks, the host-side scalar state of
+// Algorithm 1 in double precision, and the kernel launches.
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "hdet_kernels.cuh"
+#include "hdet_scalars.h"
+
+using namespace hdet;
+
+struct hdet_ctx {
+  hdet_config cfg{};
+  // schedule
+  bool has_schedule = false;
+  hdet_schedule sched{};
+  double max_lr[HDET_MAX_GROUPS]{};
+  double weight_decay[HDET_MAX_GROUPS]{};
+  // Algorithm 1 state
+  int64_t step = 0;
+  int64_t n_acc = 0;
+  bool fired = false;
+  bool round_ended = false;
+  double base[HDET_MAX_GROUPS]{};
+  double ctrl_base[HDET_MAX_GROUPS]{};
+  double velocity[HDET_MAX_GROUPS]{};
+  double delta[HDET_MAX_GROUPS]{};
+  double lr[HDET_MAX_GROUPS][HDET_MAX_REPLICAS]{};
+  double wd[HDET_MAX_GROUPS][HDET_MAX_REPLICAS]{};
+  int32_t perm_lr[HDET_MAX_GROUPS][HDET_MAX_REPLICAS]{};
+  int32_t perm_wd[HDET_MAX_GROUPS][HDET_MAX_REPLICAS]{};
+  double weights[HDET_MAX_REPLICAS]{};
+  double loss_acc[HDET_MAX_REPLICAS]{};
+  double loss_round[HDET_MAX_REPLICAS]{};
+  double rho_lr[HDET_MAX_REPLICAS]{};
+  double rho_wd[HDET_MAX_REPLICAS]{};
+  // device side
+  int64_t n_tensors = 0;
+  TensorDesc* d_tensors = nullptr;
+  Tile* d_tiles = nullptr;
+  unsigned* d_status = nullptr;
+  int n_tiles = 0;
+  int grid_fanout = 0;
+  int grid_converge = 0;
+  int64_t launches = 0;
+  std::string error;
+};
+
+namespace {
+
+thread_local std::string g_create_error;
+
+int fail(hdet_ctx* h, int code, const std::string& msg) {
+  if (h) h->error = msg; else g_create_error = msg;
+  return code;
+}
+
+int fail_cuda(hdet_ctx* h, const char* what, cudaError_t e) {
+  return fail(h, HDET_ERR_CUDA, std::string(what) + ": " + cudaGetErrorString(e));
+}
+
+bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+// Sets the handle's device for the scope of one call and restores the caller's.
+struct DeviceScope {
+  int prev = -1;
+  bool switched = false;
+  cudaError_t err = cudaSuccess;
+  explicit DeviceScope(int dev) {
+    err = cudaGetDevice(&prev);
+    if (err == cudaSuccess && prev != dev) {
+      err = cudaSetDevice(dev);
+      switched = err == cudaSuccess;
+    }
+  }
+  ~DeviceScope() { if (switched) cudaSetDevice(prev); }
+};
+
+void free_device(hdet_ctx* h) {
+  if (h->d_tensors) cudaFree(h->d_tensors);
+  if (h->d_tiles) cudaFree(h->d_tiles);
+  if (h->d_status) cudaFree(h->d_status);
+  h->d_tensors = nullptr; h->d_tiles = nullptr; h->d_status = nullptr;
+}
+
+// Rates and weight decays for the update at 0-based index h->step.
+void compute_tables(hdet_ctx* h) {
+  const int n = h->cfg.n_replicas, G = h->cfg.n_groups;
+  for (int g = 0; g < G; ++g) {
+    const double b = h->fired ? h->ctrl_base[g]
+                              : base_rate(h->sched.kind, h->step, h->sched.total_steps, h->max_lr[g],
+                                          h->sched.pct_start, h->sched.div_factor, h->sched.final_div_factor);
+    h->base[g] = b;
+    for (int r = 0; r < n; ++r) {
+      h->lr[g][r] = b * h->rho_lr[h->perm_lr[g][r]];
+      h->wd[g][r] = h->weight_decay[g] * h->rho_wd[h->perm_wd[g][r]];
+    }
+  }
+}
+
+bool is_permutation(const int32_t* p, int n) {
+  bool seen[HDET_MAX_REPLICAS] = {};
+  for (int r = 0; r < n; ++r) {
+    if (p[r] < 0 || p[r] >= n || seen[p[r]]) return false;
+    seen[p[r]] = true;
+  }
+  return true;
+}
+
+}  // namespace
+
+extern "C" {
+
+int hdet_create(const hdet_config* cfg, const hdet_tensor* tensors, int64_t n_tensors, hdet_handle* out) {
+  if (out) *out = nullptr;
+  if (!cfg || !out) return fail(nullptr, HDET_ERR_INVALID_ARG, "hdet_create: cfg and out must not be NULL");
+  if (n_tensors < 0 || (n_tensors > 0 && !tensors))
+    return fail(nullptr, HDET_ERR_INVALID_ARG, "hdet_create: tensors is NULL or n_tensors < 0");
+  if (cfg->n_replicas < 1 || cfg->n_replicas > HDET_MAX_REPLICAS)
+    return fail(nullptr, HDET_ERR_INVALID_ARG, "hdet_create: n_replicas must be in 1..32");
+  if (cfg->n_groups < 1 || cfg->n_groups > HDET_MAX_GROUPS)
+    return fail(nullptr, HDET_ERR_INVALID_ARG, "hdet_create: n_groups must be in 1..8");
+  if (cfg->optimizer != HDET_OPT_SGD && cfg->optimizer != HDET_OPT_ADAMW)
+    return fail(nullptr, HDET_ERR_INVALID_ARG, "hdet_create: unknown optimizer");
+  if (cfg->grad_dtype != HDET_DTYPE_F32 && cfg->grad_dtype != HDET_DTYPE_BF16)
+    return fail(nullptr, HDET_ERR_INVALID_ARG, "hdet_create: unknown grad_dtype");
+  if (!(cfg->alpha_lr >= 0.0 && cfg->alpha_lr < 1.0) || !(cfg->alpha_wd >= 0.0 && cfg->alpha_wd < 1.0))
+    return fail(nullptr, HDET_ERR_INVALID_ARG, "hdet_create: spread ratios must satisfy 0 <= alpha < 1");
+  if (cfg->sync_interval < 1) return fail(nullptr, HDET_ERR_INVALID_ARG, "hdet_create: sync_interval must be >= 1");
+  if (cfg->optimizer == HDET_OPT_ADAMW) {
+    if (!(cfg->beta1 >= 0.0 && cfg->beta1 < 1.0) || !(cfg->beta2 >= 0.0 && cfg->beta2 < 1.0) || !(cfg->eps >= 0.0))
+      return fail(nullptr, HDET_ERR_INVALID_ARG, "hdet_create: need 0 <= beta1, beta2 < 1 and eps >= 0");
+  }
+  if (cfg->momentum != 0.0) return fail(nullptr, HDET_ERR_UNSUPPORTED, "hdet_create: SGD momentum is not implemented");
+
+  const int n = cfg->n_replicas;
+  const size_t gsz = cfg->grad_dtype == HDET_DTYPE_BF16 ? 2 : 4;
+  std::vector<TensorDesc> descs;
+  std::vector<Tile> tiles;
+  for (int64_t k = 0; k < n_tensors; ++k) {
+    const hdet_tensor& t = tensors[k];
+    char where[64];
+    snprintf(where, sizeof where, "hdet_create: tensor %lld: ", (long long)k);
+    if (!t.param || !t.grad) return fail(nullptr, HDET_ERR_INVALID_ARG, std::string(where) + "param or grad is NULL");
+    if (cfg->optimizer == HDET_OPT_ADAMW && (!t.exp_avg || !t.exp_avg_sq))
+      return fail(nullptr, HDET_ERR_INVALID_ARG, std::string(where) + "AdamW needs exp_avg and exp_avg_sq");
+    if (t.numel <= 0) return fail(nullptr, HDET_ERR_INVALID_ARG, std::string(where) + "numel must be > 0");
+    if (t.group < 0 || t.group >= cfg->n_groups)
+      return fail(nullptr, HDET_ERR_INVALID_ARG, std::string(where) + "group out of range");
+    if (n > 1 && (t.param_stride < t.numel || (t.grad_stride != 0 && t.grad_stride < t.numel) ||
+                  (cfg->optimizer == HDET_OPT_ADAMW && t.state_stride < t.numel)))
+      return fail(nullptr, HDET_ERR_INVALID_ARG, std::string(where) + "a replica stride is smaller than numel");
+    if (t.param_stride < 0 || t.grad_stride < 0 || t.state_stride < 0)
+      return fail(nullptr, HDET_ERR_INVALID_ARG, std::string(where) + "negative stride");
+    if (!aligned(t.param, 4) || !aligned(t.grad, gsz) || (t.exp_avg && !aligned(t.exp_avg, 4)) ||
+        (t.exp_avg_sq && !aligned(t.exp_avg_sq, 4)))
+      return fail(nullptr, HDET_ERR_ALIGN, std::string(where) + "pointer not aligned to its element type");
+    const int64_t n_tiles_t = (t.numel + kTileElems - 1) / kTileElems;
+    if (n_tiles_t > INT32_MAX || (int64_t)tiles.size() + n_tiles_t > INT32_MAX)
+      return fail(nullptr, HDET_ERR_UNSUPPORTED, std::string(where) + "too many tiles");
+    TensorDesc d{};
+    d.param = static_cast<float*>(t.param);
+    d.grad = t.grad;
+    d.exp_avg = static_cast<float*>(t.exp_avg);
+    d.exp_avg_sq = static_cast<float*>(t.exp_avg_sq);
+    d.numel = t.numel;
+    d.param_stride = t.param_stride;
+    d.grad_stride = t.grad_stride;
+    d.state_stride = t.state_stride;
+    d.group = t.group;
+    bool vec = aligned(t.param, 16) && aligned(t.grad, 4 * gsz) && t.param_stride % 4 == 0 && t.grad_stride % 4 == 0;
+    if (cfg->optimizer == HDET_OPT_ADAMW)
+      vec = vec && aligned(t.exp_avg, 16) && aligned(t.exp_avg_sq, 16) && t.state_stride % 4 == 0;
+    d.vec = vec ? 1 : 0;
+    descs.push_back(d);
+    for (int64_t j = 0; j < n_tiles_t; ++j) tiles.push_back(Tile{(int)k, (int)j});
+  }
+
+  hdet_ctx* h = new (std::nothrow) hdet_ctx();
+  if (!h) return fail(nullptr, HDET_ERR_INVALID_ARG, "hdet_create: out of host memory");
+  h->cfg = *cfg;
+  h->n_tensors = n_tensors;
+  h->n_tiles = (int)tiles.size();
+  spread_multipliers(n, cfg->alpha_lr, h->rho_lr);
+  spread_multipliers(n, cfg->alpha_wd, h->rho_wd);
+  for (int g = 0; g < HDET_MAX_GROUPS; ++g)
+    for (int r = 0; r < HDET_MAX_REPLICAS; ++r) h->perm_lr[g][r] = h->perm_wd[g][r] = r;
+
+  if (n_tensors > 0) {
+    DeviceScope scope(cfg->device);
+    cudaError_t e = scope.err;
+    int sms = 0, occ_f = 0, occ_c = 0;
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, cfg->device);
+    if (e == cudaSuccess) e = fanout_occupancy(cfg->optimizer, cfg->grad_dtype, &occ_f);
+    if (e == cudaSuccess) e = converge_occupancy(&occ_c);
+    if (e == cudaSuccess) e = cudaMalloc(&h->d_tensors, descs.size() * sizeof(TensorDesc));
+    if (e == cudaSuccess) e = cudaMalloc(&h->d_tiles, tiles.size() * sizeof(Tile));
+    if (e == cudaSuccess) e = cudaMalloc(&h->d_status, sizeof(unsigned));
+    if (e == cudaSuccess) e = cudaMemcpy(h->d_tensors, descs.data(), descs.size() * sizeof(TensorDesc), cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMemcpy(h->d_tiles, tiles.data(), tiles.size() * sizeof(Tile), cudaMemcpyHostToDevice);
+    if (e == cudaSuccess) e = cudaMemset(h->d_status, 0, sizeof(unsigned));
+    if (e != cudaSuccess) {
+      free_device(h);
+      delete h;
+      return fail_cuda(nullptr, "hdet_create", e);
+    }
+    if (occ_f < 1) occ_f = 1;
+    if (occ_c < 1) occ_c = 1;
+    const int64_t cap_f = (int64_t)sms * occ_f, cap_c = (int64_t)sms * occ_c;
+    h->grid_fanout = (int)(h->n_tiles < cap_f ? h->n_tiles : cap_f);
+    h->grid_converge = (int)(h->n_tiles < cap_c ? h->n_tiles : cap_c);
+  }
+  *out = h;
+  return HDET_OK;
+}
+
+int hdet_set_schedule(hdet_handle h, const hdet_schedule* s) {
+  if (!h) return HDET_ERR_INVALID_ARG;
+  if (!s || !s->max_lr) return fail(h, HDET_ERR_INVALID_ARG, "hdet_set_schedule: sched and max_lr must not be NULL");
+  if (s->kind < HDET_SCHED_CONSTANT || s->kind > HDET_SCHED_ONECYCLE_LINEAR)
+    return fail(h, HDET_ERR_INVALID_ARG, "hdet_set_schedule: unknown kind");
+  if (s->total_steps < 1) return fail(h, HDET_ERR_INVALID_ARG, "hdet_set_schedule: total_steps must be >= 1");
+  if (s->kind != HDET_SCHED_CONSTANT) {
+    const double knee = s->pct_start * (double)s->total_steps;
+    if (!(knee > 1.0) || !(s->pct_start < 1.0))
+      return fail(h, HDET_ERR_INVALID_ARG, "hdet_set_schedule: need 1 < pct_start*total_steps and pct_start < 1");
+    if (!(s->div_factor > 0.0) || !(s->final_div_factor > 0.0))
+      return fail(h, HDET_ERR_INVALID_ARG, "hdet_set_schedule: div_factor and final_div_factor must be > 0");
+  }
+  if (s->autolr) {
+    if (!(s->sigma > 0.0)) return fail(h, HDET_ERR_INVALID_ARG, "hdet_set_schedule: sigma must be > 0");
+    if (!(s->f_div > 0.0) || !(s->f_final > 0.0))
+      return fail(h, HDET_ERR_INVALID_ARG, "hdet_set_schedule: f_div and f_final must be > 0");
+    if (s->warmup_steps < 0) return fail(h, HDET_ERR_INVALID_ARG, "hdet_set_schedule: warmup_steps must be >= 0");
+  }
+  for (int g = 0; g < h->cfg.n_groups; ++g) {
+    if (!std::isfinite(s->max_lr[g])) return fail(h, HDET_ERR_INVALID_ARG, "hdet_set_schedule: max_lr is not finite");
+    if (s->weight_decay && !std::isfinite(s->weight_decay[g]))
+      return fail(h, HDET_ERR_INVALID_ARG, "hdet_set_schedule: weight_decay is not finite");
+  }
+  h->sched = *s;
+  for (int g = 0; g < h->cfg.n_groups; ++g) {
+    h->max_lr[g] = s->max_lr[g];
+    h->weight_decay[g] = s->weight_decay ? s->weight_decay[g] : 0.0;
+  }
+  h->sched.max_lr = nullptr;
+  h->sched.weight_decay = nullptr;
+  h->has_schedule = true;
+  return HDET_OK;
+}
+
+int hdet_step(hdet_handle h, const double* step_losses, void* stream, int32_t* did_converge) {
+  if (!h) return HDET_ERR_INVALID_ARG;
+  if (did_converge) *did_converge = 0;
+  if (!h->has_schedule) return fail(h, HDET_ERR_STATE, "hdet_step: call hdet_set_schedule first");
+  const int n = h->cfg.n_replicas, G = h->cfg.n_groups;
+  compute_tables(h);
+  const int64_t t = h->step + 1;
+  const bool ends_round = (t % h->cfg.sync_interval) == 0;
+
+  if (h->n_tiles > 0) {
+    StepScalars s{};
+    const bool adam = h->cfg.optimizer == HDET_OPT_ADAMW;
+    double bc1 = 1.0, bc2 = 1.0;
+    if (adam) {
+      bc1 = 1.0 - std::pow(h->cfg.beta1, (double)t);
+      bc2 = 1.0 - std::pow(h->cfg.beta2, (double)t);
+    }
+    for (int g = 0; g < G; ++g)
+      for (int r = 0; r < n; ++r) {
+        s.decay[g][r] = adam ? (float)(1.0 - h->lr[g][r] * h->wd[g][r]) : 1.0f;
+        s.step[g][r] = (float)(adam ? h->lr[g][r] / bc1 : h->lr[g][r]);
+      }
+    s.beta1 = (float)h->cfg.beta1;
+    s.one_minus_beta1 = (float)(1.0 - h->cfg.beta1);
+    s.beta2 = (float)h->cfg.beta2;
+    s.one_minus_beta2 = (float)(1.0 - h->cfg.beta2);
+    s.rsqrt_bc2 = (float)(1.0 / std::sqrt(bc2));
+    s.eps = (float)h->cfg.eps;
+    s.inv_n = 1.0 / (double)n;
+    s.n_replicas = n;
+
+    DeviceScope scope(h->cfg.device);
+    if (scope.err != cudaSuccess) return fail_cuda(h, "hdet_step", scope.err);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const bool fuse = ends_round && h->cfg.fuse_converge;
+    LaunchPlan plan{h->d_tensors, h->d_tiles, h->n_tiles, h->grid_fanout, h->d_status};
+    cudaError_t e = launch_fanout(h->cfg.optimizer, h->cfg.grad_dtype, fuse, plan, s, st);
+    if (e != cudaSuccess) return fail_cuda(h, "hdet_step: fan-out launch", e);
+    ++h->launches;
+    if (ends_round && !fuse) {
+      plan.grid = h->grid_converge;
+      e = launch_converge(plan, n, st);
+      if (e != cudaSuccess) return fail_cuda(h, "hdet_step: converge launch", e);
+      ++h->launches;
+    }
+  }
+
+  if (step_losses)
+    for (int r = 0; r < n; ++r) h->loss_acc[r] += step_losses[r];
+  ++h->n_acc;
+  h->step = t;
+  h->round_ended = false;
+  if (ends_round) {
+    for (int r = 0; r < n; ++r) {
+      h->loss_round[r] = h->loss_acc[r] / (double)h->n_acc;
+      h->loss_acc[r] = 0.0;
+    }
+    h->n_acc = 0;
+    h->round_ended = true;
+    if (did_converge) *did_converge = 1;
+  }
+  return HDET_OK;
+}
+
+int hdet_converge(hdet_handle h, void* stream) {
+  if (!h) return HDET_ERR_INVALID_ARG;
+  if (h->n_tiles == 0) return HDET_OK;
+  DeviceScope scope(h->cfg.device);
+  if (scope.err != cudaSuccess) return fail_cuda(h, "hdet_converge", scope.err);
+  LaunchPlan plan{h->d_tensors, h->d_tiles, h->n_tiles, h->grid_converge, h->d_status};
+  cudaError_t e = launch_converge(plan, h->cfg.n_replicas, static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return fail_cuda(h, "hdet_converge: launch", e);
+  ++h->launches;
+  return HDET_OK;
+}
+
+int hdet_autolr_update(hdet_handle h, const double* round_losses, void* /*stream*/) {
+  if (!h) return HDET_ERR_INVALID_ARG;
+  if (!h->has_schedule) return fail(h, HDET_ERR_STATE, "hdet_autolr_update: call hdet_set_schedule first");
+  if (!h->round_ended)
+    return fail(h, HDET_ERR_STATE, "hdet_autolr_update: the last hdet_step did not end a round (or the update already ran)");
+  h->round_ended = false;
+  if (!h->sched.autolr || h->step < h->sched.warmup_steps) return HDET_OK;
+  const int n = h->cfg.n_replicas, G = h->cfg.n_groups;
+  const double* L = round_losses ? round_losses : h->loss_round;
+  for (int r = 0; r < n; ++r)
+    if (!std::isfinite(L[r])) {
+      h->round_ended = true;
+      return fail(h, HDET_ERR_INVALID_ARG, "hdet_autolr_update: a round loss is not finite");
+    }
+  if (round_losses)
+    for (int r = 0; r < n; ++r) h->loss_round[r] = round_losses[r];
+  const double gamma = decay_gamma(h->sched.f_div, h->sched.f_final, h->sched.total_steps, h->sched.warmup_steps,
+                                   h->cfg.sync_interval);
+  softmax_weights(n, L, h->sched.sigma, h->weights);                       // Eq. 4
+  for (int g = 0; g < G; ++g) {
+    double weighted = 0.0, plain = 0.0;
+    for (int r = 0; r < n; ++r) {
+      weighted += h->weights[r] * h->lr[g][r];                             // Eq. 5
+      plain += h->lr[g][r];
+    }
+    plain /= n;
+    h->delta[g] = weighted - plain;                                        // Eq. 6
+    h->velocity[g] = h->sched.beta * h->velocity[g] + (1.0 - h->sched.beta) * h->delta[g];   // Eq. 7
+    h->ctrl_base[g] = plain * (1.0 - gamma) + h->velocity[g] * h->sched.lambda;
+  }
+  h->fired = true;
+  if (h->cfg.reshuffle) {                                                   // Eq. 9
+    const uint64_t sync_index = (uint64_t)(h->step / h->cfg.sync_interval);
+    for (int g = 0; g < G; ++g) {
+      draw_permutation(h->cfg.seed, sync_index, 2ull * g, n, h->perm_lr[g]);
+      draw_permutation(h->cfg.seed, sync_index, 2ull * g + 1, n, h->perm_wd[g]);
+    }
+  }
+  return HDET_OK;
+}
+
+int hdet_get_state(hdet_handle h, hdet_state* out) {
+  if (!h) return HDET_ERR_INVALID_ARG;
+  if (!out) return fail(h, HDET_ERR_INVALID_ARG, "hdet_get_state: out is NULL");
+  std::memset(out, 0, sizeof *out);
+  out->step = h->step;
+  out->n_acc = h->n_acc;
+  out->fired = h->fired;
+  out->round_ended = h->round_ended;
+  std::memcpy(out->base, h->base, sizeof h->base);
+  std::memcpy(out->ctrl_base, h->ctrl_base, sizeof h->ctrl_base);
+  std::memcpy(out->velocity, h->velocity, sizeof h->velocity);
+  std::memcpy(out->delta, h->delta, sizeof h->delta);
+  std::memcpy(out->lr, h->lr, sizeof h->lr);
+  std::memcpy(out->wd, h->wd, sizeof h->wd);
+  std::memcpy(out->perm_lr, h->perm_lr, sizeof h->perm_lr);
+  std::memcpy(out->perm_wd, h->perm_wd, sizeof h->perm_wd);
+  std::memcpy(out->weights, h->weights, sizeof h->weights);
+  std::memcpy(out->loss_acc, h->loss_acc, sizeof h->loss_acc);
+  std::memcpy(out->loss_round, h->loss_round, sizeof h->loss_round);
+  out->gamma = h->has_schedule ? decay_gamma(h->sched.f_div, h->sched.f_final, h->sched.total_steps,
+                                             h->sched.warmup_steps, h->cfg.sync_interval)
+                               : 0.0;
+  if (h->d_status) {
+    DeviceScope scope(h->cfg.device);
+    cudaError_t e = scope.err;
+    unsigned word = 0;
+    if (e == cudaSuccess) e = cudaMemcpy(&word, h->d_status, sizeof word, cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return fail_cuda(h, "hdet_get_state", e);
+    out->device_status = word;
+    if (word & 1u) return fail(h, HDET_ERR_NONFINITE, "a kernel produced a non-finite parameter");
+  }
+  return HDET_OK;
+}
+
+int hdet_set_state(hdet_handle h, const hdet_state* in) {
+  if (!h) return HDET_ERR_INVALID_ARG;
+  if (!in) return fail(h, HDET_ERR_INVALID_ARG, "hdet_set_state: in is NULL");
+  if (in->step < 0 || in->n_acc < 0) return fail(h, HDET_ERR_INVALID_ARG, "hdet_set_state: negative step or n_acc");
+  const int n = h->cfg.n_replicas, G = h->cfg.n_groups;
+  for (int g = 0; g < G; ++g)
+    if (!is_permutation(in->perm_lr[g], n) || !is_permutation(in->perm_wd[g], n))
+      return fail(h, HDET_ERR_INVALID_ARG, "hdet_set_state: a permutation array is not a permutation of 0..N-1");
+  h->step = in->step;
+  h->n_acc = in->n_acc;
+  h->fired = in->fired != 0;
+  h->round_ended = in->round_ended != 0;
+  std::memcpy(h->ctrl_base, in->ctrl_base, sizeof h->ctrl_base);
+  std::memcpy(h->velocity, in->velocity, sizeof h->velocity);
+  std::memcpy(h->lr, in->lr, sizeof h->lr);  // rates of the last update: Eq. 5 needs them if a round just ended
+  for (int g = 0; g < G; ++g) {
+    std::memcpy(h->perm_lr[g], in->perm_lr[g], sizeof(int32_t) * n);
+    std::memcpy(h->perm_wd[g], in->perm_wd[g], sizeof(int32_t) * n);
+  }
+  std::memcpy(h->loss_acc, in->loss_acc, sizeof h->loss_acc);
+  std::memcpy(h->loss_round, in->loss_round, sizeof h->loss_round);
+  if (h->d_status) {
+    DeviceScope scope(h->cfg.device);
+    cudaError_t e = scope.err;
+    if (e == cudaSuccess) e = cudaMemset(h->d_status, 0, sizeof(unsigned));
+    if (e != cudaSuccess) return fail_cuda(h, "hdet_set_state", e);
+  }
+  return HDET_OK;
+}
+
+int hdet_destroy(hdet_handle h) {
+  if (!h) return HDET_OK;
+  if (h->d_tensors || h->d_tiles || h->d_status) {
+    DeviceScope scope(h->cfg.device);
+    free_device(h);
+  }
+  delete h;
+  return HDET_OK;
+}
+
+const char* hdet_last_error(hdet_handle h) { return h ? h->error.c_str() : g_create_error.c_str(); }
+
+int64_t hdet_kernel_launches(hdet_handle h) { return h ? h->launches : 0; }
+
+}  // extern "C"

@@ -1,0 +1,309 @@
+// Fan-out update and converge kernels for sm_100a.
+//
+// Work assignment: one CTA owns one tile (kTileElems consecutive elements of one tensor)
+// and streams ALL N replicas of that tile, so the replica mean of Eq. 3 is a per-thread
+// register accumulation: no inter-CTA dependence, no atomics on data, no device-side wait.
+// The path is HBM-bound (about 1.5 flop per byte): accesses are 128-bit, warp-contiguous,
+// read-once / write-once with streaming cache hints, and replica r+1 is loaded while
+// replica r is being computed and stored (explicit two-stage register pipeline).
+#include <cuda_bf16.h>
+
+#include <type_traits>
+
+#include "hdet_kernels.cuh"
+
+namespace hdet {
+namespace {
+
+struct AdamConsts {
+  float beta1, one_minus_beta1, beta2, one_minus_beta2, rsqrt_bc2, eps;
+};
+
+// Adam with decoupled weight decay on one element (Section 4.1 names Adam; weight decay is a
+// spreadable scalar per Remark 1):
+//   theta *= 1 - lr*wd ; m = b1 m + (1-b1) g ; v = b2 v + (1-b2) g^2 ;
+//   theta -= lr/(1-b1^t) * m / (sqrt(v)/sqrt(1-b2^t) + eps)
+__device__ __forceinline__ void adam_element(float& th, float& m, float& v, float g, float decay, float step,
+                                             const AdamConsts& c) {
+  m = fmaf(c.beta1, m, c.one_minus_beta1 * g);
+  v = fmaf(c.beta2, v, c.one_minus_beta2 * g * g);
+  const float denom = fmaf(sqrtf(v), c.rsqrt_bc2, c.eps);
+  th = fmaf(-step, m / denom, th * decay);
+}
+
+// Eq. 2: theta <- theta - eta_r * g
+__device__ __forceinline__ void sgd_element(float& th, float g, float step) { th = fmaf(-step, g, th); }
+
+__device__ __forceinline__ bool not_finite(float x) { return !(fabsf(x) <= 3.402823466e38f); }
+
+// ---- gradient access: fp32 (float4 per 4 elements) or bf16 (uint2 per 4 elements) ----------
+template <typename GradT> struct GradRaw;
+template <> struct GradRaw<float> { using type = float4; };
+template <> struct GradRaw<__nv_bfloat16> { using type = uint2; };
+
+__device__ __forceinline__ float4 load_raw(const float* p) { return __ldcs(reinterpret_cast<const float4*>(p)); }
+__device__ __forceinline__ uint2 load_raw(const __nv_bfloat16* p) { return __ldcs(reinterpret_cast<const uint2*>(p)); }
+__device__ __forceinline__ void unpack(const float4& r, float (&g)[4]) { g[0] = r.x; g[1] = r.y; g[2] = r.z; g[3] = r.w; }
+__device__ __forceinline__ void unpack(const uint2& r, float (&g)[4]) {
+  g[0] = __uint_as_float(r.x << 16);
+  g[1] = __uint_as_float(r.x & 0xffff0000u);
+  g[2] = __uint_as_float(r.y << 16);
+  g[3] = __uint_as_float(r.y & 0xffff0000u);
+}
+__device__ __forceinline__ float load_scalar(const float* p) { return __ldcs(p); }
+__device__ __forceinline__ float load_scalar(const __nv_bfloat16* p) {
+  return __uint_as_float(static_cast<unsigned>(__ldcs(reinterpret_cast<const unsigned short*>(p))) << 16);
+}
+
+// ---- scalar path: elements [begin, end) of one tensor, any alignment -----------------------
+template <typename GradT, bool kAdam, bool kConv>
+__device__ void range_scalar(const TensorDesc& td, long long begin, long long end, const StepScalars& s,
+                             const AdamConsts& c, bool& bad) {
+  const int n = s.n_replicas;
+  const GradT* grad = static_cast<const GradT*>(td.grad);
+  for (long long e = begin + threadIdx.x; e < end; e += kThreads) {
+    double sum = 0.0;
+    for (int r = 0; r < n; ++r) {
+      float th = __ldcs(td.param + r * td.param_stride + e);
+      const float g = load_scalar(grad + r * td.grad_stride + e);
+      if (kAdam) {
+        float m = __ldcs(td.exp_avg + r * td.state_stride + e);
+        float v = __ldcs(td.exp_avg_sq + r * td.state_stride + e);
+        adam_element(th, m, v, g, s.decay[td.group][r], s.step[td.group][r], c);
+        __stcs(td.exp_avg + r * td.state_stride + e, m);
+        __stcs(td.exp_avg_sq + r * td.state_stride + e, v);
+      } else {
+        sgd_element(th, g, s.step[td.group][r]);
+      }
+      bad |= not_finite(th);
+      if (kConv) sum += (double)th;
+      else __stcs(td.param + r * td.param_stride + e, th);
+    }
+    if (kConv) {
+      const float mean = (float)(sum * s.inv_n);
+      for (int r = 0; r < n; ++r) __stcs(td.param + r * td.param_stride + e, mean);
+    }
+  }
+}
+
+// ---- vector path ---------------------------------------------------------------------------
+template <typename GradT, bool kAdam>
+struct ReplicaRegs {
+  float4 th[kTileVecs];
+  float4 m[kAdam ? kTileVecs : 1];
+  float4 v[kAdam ? kTileVecs : 1];
+  typename GradRaw<GradT>::type g[kTileVecs];
+};
+
+// Processes `nvec` float4 vectors starting at element `off` of the tensor.  kFull: nvec == kThreads*kTileVecs.
+template <typename GradT, bool kAdam, bool kConv, bool kFull>
+__device__ __forceinline__ void tile_vector(const TensorDesc& td, long long off, int nvec, const StepScalars& s,
+                                            const AdamConsts& c, bool& bad) {
+  using Regs = ReplicaRegs<GradT, kAdam>;
+  const int n = s.n_replicas;
+  const int grp = td.group;
+  float* const P = td.param + off;
+  float* const M = kAdam ? td.exp_avg + off : nullptr;
+  float* const V = kAdam ? td.exp_avg_sq + off : nullptr;
+  const GradT* const Gp = static_cast<const GradT*>(td.grad) + off;
+  const long long ps = td.param_stride, gs = td.grad_stride, ss = td.state_stride;
+
+  int idx[kTileVecs];
+  bool ok[kTileVecs];
+#pragma unroll
+  for (int k = 0; k < kTileVecs; ++k) {
+    const int j = k * kThreads + threadIdx.x;
+    idx[k] = j * 4;
+    ok[k] = kFull || j < nvec;
+  }
+
+  auto load = [&](Regs& b, int r) {
+#pragma unroll
+    for (int k = 0; k < kTileVecs; ++k) {
+      if (ok[k]) {
+        b.th[k] = __ldcs(reinterpret_cast<const float4*>(P + r * ps + idx[k]));
+        if (kAdam) {
+          b.m[k] = __ldcs(reinterpret_cast<const float4*>(M + r * ss + idx[k]));
+          b.v[k] = __ldcs(reinterpret_cast<const float4*>(V + r * ss + idx[k]));
+        }
+        b.g[k] = load_raw(Gp + r * gs + idx[k]);
+      } else {
+        b.th[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (kAdam) { b.m[k] = b.th[k]; b.v[k] = b.th[k]; }
+        b.g[k] = typename GradRaw<GradT>::type{};
+      }
+    }
+  };
+
+  double sum[kConv ? kTileVecs : 1][4];
+  if (kConv) {
+#pragma unroll
+    for (int k = 0; k < kTileVecs; ++k)
+#pragma unroll
+      for (int q = 0; q < 4; ++q) sum[k][q] = 0.0;
+  }
+
+  auto update_store = [&](Regs& b, int r) {
+    const float decay = s.decay[grp][r];
+    const float step = s.step[grp][r];
+#pragma unroll
+    for (int k = 0; k < kTileVecs; ++k) {
+      float g[4];
+      unpack(b.g[k], g);
+      float th[4] = {b.th[k].x, b.th[k].y, b.th[k].z, b.th[k].w};
+      if (kAdam) {
+        float m[4] = {b.m[k].x, b.m[k].y, b.m[k].z, b.m[k].w};
+        float v[4] = {b.v[k].x, b.v[k].y, b.v[k].z, b.v[k].w};
+#pragma unroll
+        for (int q = 0; q < 4; ++q) adam_element(th[q], m[q], v[q], g[q], decay, step, c);
+        if (ok[k]) {
+          __stcs(reinterpret_cast<float4*>(M + r * ss + idx[k]), make_float4(m[0], m[1], m[2], m[3]));
+          __stcs(reinterpret_cast<float4*>(V + r * ss + idx[k]), make_float4(v[0], v[1], v[2], v[3]));
+        }
+      } else {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) sgd_element(th[q], g[q], step);
+      }
+#pragma unroll
+      for (int q = 0; q < 4; ++q) bad |= not_finite(th[q]);
+      if (kConv) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) sum[k][q] += (double)th[q];
+      } else if (ok[k]) {
+        __stcs(reinterpret_cast<float4*>(P + r * ps + idx[k]), make_float4(th[0], th[1], th[2], th[3]));
+      }
+    }
+  };
+
+  // Two-stage register pipeline over the replica axis.
+  Regs a, b;
+  load(a, 0);
+  int r = 0;
+  for (; r + 1 < n; r += 2) {
+    load(b, r + 1);
+    update_store(a, r);
+    if (r + 2 < n) load(a, r + 2);
+    update_store(b, r + 1);
+  }
+  if (r < n) update_store(a, r);
+
+  if (kConv) {
+    // Eq. 3: the mean of the updated replicas goes to every replica.
+#pragma unroll
+    for (int k = 0; k < kTileVecs; ++k) {
+      if (!ok[k]) continue;
+      const float4 mean = make_float4((float)(sum[k][0] * s.inv_n), (float)(sum[k][1] * s.inv_n),
+                                      (float)(sum[k][2] * s.inv_n), (float)(sum[k][3] * s.inv_n));
+      for (int rr = 0; rr < n; ++rr) __stcs(reinterpret_cast<float4*>(P + rr * ps + idx[k]), mean);
+    }
+  }
+}
+
+template <typename GradT, bool kAdam, bool kConv>
+__global__ void __launch_bounds__(kThreads, 2)
+fanout_kernel(const __grid_constant__ LaunchPlan plan, const __grid_constant__ StepScalars s) {
+  const AdamConsts c{s.beta1, s.one_minus_beta1, s.beta2, s.one_minus_beta2, s.rsqrt_bc2, s.eps};
+  bool bad = false;
+  for (int t = blockIdx.x; t < plan.n_tiles; t += gridDim.x) {
+    const Tile tile = plan.tiles[t];
+    const TensorDesc td = plan.tensors[tile.tensor];
+    const long long off = (long long)tile.tile * kTileElems;
+    const long long rest = td.numel - off;
+    const int len = rest < kTileElems ? (int)rest : kTileElems;
+    if (td.vec) {
+      if (len == kTileElems) {
+        tile_vector<GradT, kAdam, kConv, true>(td, off, kThreads * kTileVecs, s, c, bad);
+      } else {
+        const int nvec = len >> 2;
+        if (nvec) tile_vector<GradT, kAdam, kConv, false>(td, off, nvec, s, c, bad);
+        if (len & 3) range_scalar<GradT, kAdam, kConv>(td, off + 4ll * nvec, off + len, s, c, bad);
+      }
+    } else {
+      range_scalar<GradT, kAdam, kConv>(td, off, off + len, s, c, bad);
+    }
+  }
+  if (bad) atomicOr(plan.status, 1u);
+}
+
+// ---- stand-alone converge (Eq. 3) -------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads, 4)
+converge_kernel(const __grid_constant__ LaunchPlan plan, int n, double inv_n) {
+  for (int t = blockIdx.x; t < plan.n_tiles; t += gridDim.x) {
+    const Tile tile = plan.tiles[t];
+    const TensorDesc td = plan.tensors[tile.tensor];
+    const long long off = (long long)tile.tile * kTileElems;
+    const long long rest = td.numel - off;
+    const int len = rest < kTileElems ? (int)rest : kTileElems;
+    const int nvec = td.vec ? (len >> 2) : 0;
+    float* const P = td.param + off;
+    for (int j = threadIdx.x; j < nvec; j += kThreads) {
+      double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
+#pragma unroll 4
+      for (int r = 0; r < n; ++r) {
+        const float4 x = __ldcs(reinterpret_cast<const float4*>(P + r * td.param_stride + 4 * j));
+        s0 += (double)x.x; s1 += (double)x.y; s2 += (double)x.z; s3 += (double)x.w;
+      }
+      const float4 mean = make_float4((float)(s0 * inv_n), (float)(s1 * inv_n), (float)(s2 * inv_n), (float)(s3 * inv_n));
+      for (int r = 0; r < n; ++r) __stcs(reinterpret_cast<float4*>(P + r * td.param_stride + 4 * j), mean);
+    }
+    for (int e = 4 * nvec + threadIdx.x; e < len; e += kThreads) {
+      double sum = 0.0;
+      for (int r = 0; r < n; ++r) sum += (double)__ldcs(P + r * td.param_stride + e);
+      const float mean = (float)(sum * inv_n);
+      for (int r = 0; r < n; ++r) __stcs(P + r * td.param_stride + e, mean);
+    }
+  }
+}
+
+template <typename GradT, bool kAdam, bool kConv>
+cudaError_t launch_one(const LaunchPlan& plan, const StepScalars& s, cudaStream_t stream) {
+  fanout_kernel<GradT, kAdam, kConv><<<plan.grid, kThreads, 0, stream>>>(plan, s);
+  return cudaGetLastError();
+}
+
+template <typename GradT, bool kAdam>
+cudaError_t occupancy_one(int* out) {
+  int a = 0, b = 0;
+  cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&a, fanout_kernel<GradT, kAdam, false>, kThreads, 0);
+  if (e != cudaSuccess) return e;
+  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, fanout_kernel<GradT, kAdam, true>, kThreads, 0);
+  if (e != cudaSuccess) return e;
+  *out = a < b ? a : b;
+  return cudaSuccess;
+}
+
+}  // namespace
+
+cudaError_t launch_fanout(int optimizer, int grad_dtype, bool converge, const LaunchPlan& plan,
+                          const StepScalars& s, cudaStream_t stream) {
+  if (plan.n_tiles == 0) return cudaSuccess;
+  const bool adam = optimizer == HDET_OPT_ADAMW;
+  const bool bf16 = grad_dtype == HDET_DTYPE_BF16;
+  if (adam) {
+    if (bf16) return converge ? launch_one<__nv_bfloat16, true, true>(plan, s, stream)
+                              : launch_one<__nv_bfloat16, true, false>(plan, s, stream);
+    return converge ? launch_one<float, true, true>(plan, s, stream) : launch_one<float, true, false>(plan, s, stream);
+  }
+  if (bf16) return converge ? launch_one<__nv_bfloat16, false, true>(plan, s, stream)
+                            : launch_one<__nv_bfloat16, false, false>(plan, s, stream);
+  return converge ? launch_one<float, false, true>(plan, s, stream) : launch_one<float, false, false>(plan, s, stream);
+}
+
+cudaError_t launch_converge(const LaunchPlan& plan, int n_replicas, cudaStream_t stream) {
+  if (plan.n_tiles == 0) return cudaSuccess;
+  converge_kernel<<<plan.grid, kThreads, 0, stream>>>(plan, n_replicas, 1.0 / (double)n_replicas);
+  return cudaGetLastError();
+}
+
+cudaError_t fanout_occupancy(int optimizer, int grad_dtype, int* ctas_per_sm) {
+  const bool adam = optimizer == HDET_OPT_ADAMW;
+  const bool bf16 = grad_dtype == HDET_DTYPE_BF16;
+  if (adam) return bf16 ? occupancy_one<__nv_bfloat16, true>(ctas_per_sm) : occupancy_one<float, true>(ctas_per_sm);
+  return bf16 ? occupancy_one<__nv_bfloat16, false>(ctas_per_sm) : occupancy_one<float, false>(ctas_per_sm);
+}
+
+cudaError_t converge_occupancy(int* ctas_per_sm) {
+  return cudaOccupancyMaxActiveBlocksPerMultiprocessor(ctas_per_sm, converge_kernel, kThreads, 0);
+}
+
+}  // namespace hdet

@@ -1,0 +1,67 @@
+// Device-side data structures and launchers of the fan-out / converge kernels.
+#pragma once
+#include <cuda_runtime.h>
+
+#include <cstdint>
+
+#include "../../include/hdet.h"
+
+namespace hdet {
+
+// One tile = kTileVecs float4 vectors per thread of a kThreads-wide CTA.
+constexpr int kThreads = 256;
+constexpr int kTileVecs = 2;
+constexpr int kTileElems = kThreads * 4 * kTileVecs;  // 2048 elements
+
+// Per-tensor descriptor, resident on the device (built once by hdet_create).
+struct TensorDesc {
+  float* param;
+  const void* grad;
+  float* exp_avg;
+  float* exp_avg_sq;
+  long long numel;
+  long long param_stride;
+  long long grad_stride;
+  long long state_stride;
+  int group;
+  int vec;  // 1: pointers and strides allow 128-bit accesses
+};
+
+// One unit of work: tile `tile` (kTileElems elements) of tensor `tensor`.
+struct Tile {
+  int tensor;
+  int tile;
+};
+
+// Per-launch scalars, passed by value as kernel parameters (no device table to update).
+struct StepScalars {
+  float decay[HDET_MAX_GROUPS][HDET_MAX_REPLICAS];  // 1 - lr*wd
+  float step[HDET_MAX_GROUPS][HDET_MAX_REPLICAS];   // AdamW: lr / (1 - beta1^t); SGD: lr
+  float beta1, one_minus_beta1, beta2, one_minus_beta2;
+  float rsqrt_bc2;  // 1 / sqrt(1 - beta2^t)
+  float eps;
+  double inv_n;     // 1 / N
+  int n_replicas;
+};
+
+struct LaunchPlan {
+  const TensorDesc* tensors;
+  const Tile* tiles;
+  int n_tiles;
+  int grid;            // CTAs to launch (persistent, grid-stride over tiles)
+  unsigned* status;    // device status word; bit 0 = non-finite parameter seen
+};
+
+// Fan-out update of every replica of every tile (Eq. 2 or Adam); with `converge` the
+// replica mean (Eq. 3) is formed from the updated values and written to all replicas.
+cudaError_t launch_fanout(int optimizer, int grad_dtype, bool converge, const LaunchPlan& plan,
+                          const StepScalars& s, cudaStream_t stream);
+
+// Stand-alone Eq. 3.
+cudaError_t launch_converge(const LaunchPlan& plan, int n_replicas, cudaStream_t stream);
+
+// Resident CTAs per SM of the fan-out kernels (minimum over the variants of one optimizer/dtype).
+cudaError_t fanout_occupancy(int optimizer, int grad_dtype, int* ctas_per_sm);
+cudaError_t converge_occupancy(int* ctas_per_sm);
+
+}  // namespace hdet

@@ -24,3 +24,13 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(scope="session", autouse=True)
+def _built_libraries():
+    """Compiles the CUDA libraries in-tree when they are missing or older than their sources."""
+    from hdet_inputs import device
+    from paper_2604_24708_b200 import build
+
+    build.build()
+    device.build()

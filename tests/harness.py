@@ -1,0 +1,196 @@
+"""Shared test harness: drives the CUDA library and the CPU oracle with the same seeded inputs."""
+from __future__ import annotations
+
+from typing import List, Optional, Sequence, Tuple
+
+import numpy as np
+
+from hdet_inputs import recipes as R
+from hdet_inputs import workloads as W
+from oracle import hdet_oracle as O
+
+
+# ----------------------------------------------------------------------------- library side
+def lib_config(B, w: W.Workload, fuse: int = 1, device: int = 0):
+    return B.hdet_config(
+        n_replicas=w.n_replicas, n_groups=w.n_groups, optimizer=w.optimizer, grad_dtype=w.grad_dtype,
+        beta1=w.beta1, beta2=w.beta2, eps=w.eps, momentum=0.0, alpha_lr=w.alpha_lr, alpha_wd=w.alpha_wd,
+        sync_interval=w.sync_interval, reshuffle=w.reshuffle, fuse_converge=fuse, seed=w.seed, device=device)
+
+
+def lib_schedule(B, w: W.Workload):
+    return B.make_schedule(
+        w.sched_kind, w.total_steps, list(w.max_lr), list(w.weight_decay), pct_start=w.pct_start,
+        div_factor=w.div_factor, final_div_factor=w.final_div_factor, autolr=w.autolr,
+        warmup_steps=w.warmup_steps, beta=w.ctrl_beta, sigma=w.ctrl_sigma, lambda_=w.ctrl_lambda,
+        f_div=w.f_div, f_final=w.f_final)
+
+
+class GpuRun:
+    """The workload resident on the GPU, stepped through the C ABI."""
+
+    def __init__(self, w: W.Workload, fuse: int = 1, shared_grad: bool = False, device: int = 0):
+        import torch
+        from hdet_inputs import device as D
+        from paper_2604_24708_b200 import binding as B
+        from paper_2604_24708_b200.arena import StackedArena
+
+        self.B, self.D, self.torch, self.w = B, D, torch, w
+        self.arena = StackedArena([t.numel for t in w.tensors], [t.group for t in w.tensors], w.n_replicas,
+                                  w.optimizer, w.grad_dtype, device=f"cuda:{device}", align_elems=w.align_elems,
+                                  shared_grad=shared_grad)
+        assert self.arena.offsets == w.arena_offsets()
+        D.fill(self.arena.param[0], R.param_key(w), 0, R.param_scale(w))
+        for r in range(1, w.n_replicas):
+            self.arena.param[r].copy_(self.arena.param[0])
+        self.h = B.hdet_create(lib_config(B, w, fuse, device), self.arena.descriptors())
+        B.hdet_set_schedule(self.h, lib_schedule(B, w))
+        self.i = 0
+
+    def fill_grads(self, step: int) -> None:
+        a, w = self.arena, self.w
+        if a.shared_grad:
+            self.D.fill(a.grad, R.grad_key(w, step, 0), 0, R.grad_scale(w))
+        else:
+            for r in range(w.n_replicas):
+                self.D.fill(a.grad[r], R.grad_key(w, step, r), 0, R.grad_scale(w))
+
+    def perm0(self) -> List[int]:
+        st = self.B.hdet_get_state(self.h)
+        return list(st.perm_lr[0])[: self.w.n_replicas]
+
+    def step(self, perm0: Optional[Sequence[int]] = None) -> bool:
+        """One update with regenerated gradients and recipe losses; runs the controller after a sync."""
+        self.fill_grads(self.i)
+        losses = R.step_losses(self.w, self.i, perm0)
+        ended = self.B.hdet_step(self.h, list(losses))
+        if ended:
+            self.B.hdet_autolr_update(self.h)
+        self.i += 1
+        return ended
+
+    def state(self):
+        return self.B.hdet_get_state(self.h)
+
+    def slab(self, which: str, k: int, start: int, n: int) -> np.ndarray:
+        """[N, n] values of tensor k, elements start .. start+n-1, copied to the host."""
+        t = {"param": self.arena.param, "m": self.arena.exp_avg, "v": self.arena.exp_avg_sq}[which]
+        off = self.arena.offsets[k] + start
+        return t[:, off:off + n].float().cpu().numpy()
+
+    def close(self) -> None:
+        self.torch.cuda.synchronize()
+        self.B.hdet_destroy(self.h)
+        self.h = None
+
+
+# ----------------------------------------------------------------------------- oracle side
+Slab = Tuple[int, int, int]   # (tensor index, first element inside the tensor, length)
+
+
+def oracle_for(w: W.Workload, params: Sequence[np.ndarray], groups: Sequence[int]) -> O.HdetOracle:
+    return O.HdetOracle(
+        params, groups, w.n_groups, optimizer=w.optimizer, total_steps=w.total_steps, sched_kind=w.sched_kind,
+        max_lr=list(w.max_lr), weight_decay=list(w.weight_decay), pct_start=w.pct_start, div_factor=w.div_factor,
+        final_div_factor=w.final_div_factor, alpha_lr=w.alpha_lr, alpha_wd=w.alpha_wd,
+        sync_interval=w.sync_interval, autolr=bool(w.autolr), warmup_steps=w.warmup_steps, ctrl_beta=w.ctrl_beta,
+        ctrl_sigma=w.ctrl_sigma, ctrl_lambda=w.ctrl_lambda, f_div=w.f_div, f_final=w.f_final,
+        reshuffle=bool(w.reshuffle), seed=w.seed, beta1=w.beta1, beta2=w.beta2, eps=w.eps, n_replicas=w.n_replicas)
+
+
+class OracleRun:
+    """The oracle over chosen element ranges (slabs) of the workload, with the same seeded inputs."""
+
+    def __init__(self, w: W.Workload, slabs: Sequence[Slab], shared_grad: bool = False):
+        self.w, self.slabs, self.shared_grad = w, list(slabs), shared_grad
+        offs = w.arena_offsets()
+        self.starts = [offs[k] + s for (k, s, n) in self.slabs]
+        params = [np.tile(R.param_slab(w, a, n).astype(np.float64), (w.n_replicas, 1))
+                  for a, (k, s, n) in zip(self.starts, self.slabs)]
+        self.o = oracle_for(w, params, [w.tensors[k].group for (k, s, n) in self.slabs])
+        self.i = 0
+
+    def grads(self, step: int) -> List[np.ndarray]:
+        w = self.w
+        out = []
+        for a, (k, s, n) in zip(self.starts, self.slabs):
+            if self.shared_grad:
+                out.append(R.grad_slab(w, step, 0, a, n).astype(np.float64))
+            else:
+                out.append(np.stack([R.grad_slab(w, step, r, a, n) for r in range(w.n_replicas)]).astype(np.float64))
+        return out
+
+    def step(self) -> bool:
+        losses = R.step_losses(self.w, self.i, self.o.perm_lr[0])
+        ended = self.o.step(self.grads(self.i), losses)
+        self.i += 1
+        return ended
+
+
+def whole_tensor_slabs(w: W.Workload) -> List[Slab]:
+    return [(k, 0, t.numel) for k, t in enumerate(w.tensors)]
+
+
+def sampled_slabs(w: W.Workload, tile: int = 2048, extra: int = 2, seed: int = 0) -> List[Slab]:
+    """First and last tile of every tensor (tails included) plus `extra` random tiles of each large tensor."""
+    rng = np.random.default_rng(seed)
+    out: List[Slab] = []
+    for k, t in enumerate(w.tensors):
+        n = t.numel
+        if n <= 2 * tile:
+            out.append((k, 0, n))
+            continue
+        out.append((k, 0, tile))
+        last = max(tile, (n - 1) // tile * tile - tile)      # the last full tile together with the ragged tail
+        out.append((k, last, n - last))
+        n_tiles = n // tile
+        for j in rng.choice(np.arange(1, max(2, n_tiles - 1)), size=min(extra, max(0, n_tiles - 2)), replace=False):
+            out.append((k, int(j) * tile, tile))
+    return out
+
+
+# ----------------------------------------------------------------------------- comparison
+def rel_err(got: np.ndarray, ref: np.ndarray) -> np.ndarray:
+    """|got - ref| / max(|ref|, RMS(ref)): per-element relative error with an RMS floor near zero."""
+    ref = np.asarray(ref, dtype=np.float64)
+    rms = float(np.sqrt(np.mean(ref * ref)))
+    den = np.maximum(np.abs(ref), rms if rms > 0 else 1.0)
+    return np.abs(np.asarray(got, dtype=np.float64) - ref) / den
+
+
+def compare_slabs(g: GpuRun, o: OracleRun, tol: float, check_moments: bool = True) -> float:
+    """Largest relative error over all slabs (params and, for AdamW, both moments); asserts it is <= tol."""
+    worst = 0.0
+    adam = g.w.optimizer == W.OPT_ADAMW
+    for idx, (k, s, n) in enumerate(o.slabs):
+        pairs = [("param", o.o.theta[idx])]
+        if adam and check_moments:
+            pairs += [("m", o.o.m[idx]), ("v", o.o.v[idx])]
+        for name, ref in pairs:
+            e = rel_err(g.slab(name, k, s, n), ref).max()
+            assert e <= tol, f"{name} of tensor {k} [{s}:{s + n}] at step {g.i}: rel err {e:.3e} > {tol:.1e}"
+            worst = max(worst, float(e))
+    return worst
+
+
+def compare_scalars(st, o: O.HdetOracle, n: int, G: int, tol: float = 1e-12) -> None:
+    """Schedule / spread / controller scalars of the library against the oracle (relative 1e-12)."""
+    def close(a, b, what):
+        a, b = float(a), float(b)
+        assert abs(a - b) <= tol * max(abs(b), 1e-300) or abs(a - b) < 1e-300, f"{what}: {a!r} vs {b!r}"
+    for g in range(G):
+        close(st.base[g], o.base[g], f"base[{g}]")
+        assert abs(float(st.velocity[g]) - o.vel[g]) <= tol * max(abs(o.base[g]), 1e-300), f"velocity[{g}]"
+        if o.fired:
+            close(st.ctrl_base[g], o.ctrl_base[g], f"ctrl_base[{g}]")
+            a, b = float(st.delta[g]), float(o.delta[g])
+            assert abs(a - b) <= tol * max(abs(o.base[g]), 1e-300), f"delta[{g}]: {a!r} vs {b!r}"
+        for r in range(n):
+            close(st.lr[g][r], o.lr[g][r], f"lr[{g}][{r}]")
+            close(st.wd[g][r], o.wd[g][r], f"wd[{g}][{r}]")
+        assert list(st.perm_lr[g])[:n] == o.perm_lr[g], f"perm_lr[{g}]"
+        assert list(st.perm_wd[g])[:n] == o.perm_wd[g], f"perm_wd[{g}]"
+    assert bool(st.fired) == o.fired
+    if o.w is not None:
+        for r in range(n):
+            close(st.weights[r], o.w[r], f"w[{r}]")

@@ -1,0 +1,230 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle on the same seeded inputs.
+
+Tolerances (relative error per element with denominator max(|oracle|, RMS of the oracle slab)):
+1e-6 after one update, 1e-5 after a full run; schedule and controller scalars 1e-12.
+"""
+from dataclasses import replace
+
+import numpy as np
+import pytest
+
+import harness as H
+from hdet_inputs import generator as G
+from hdet_inputs import recipes as R
+from hdet_inputs import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+TOL_ONE_STEP = 1e-6
+TOL_FULL_RUN = 1e-5
+
+
+def _lockstep(w, slabs, steps=None, fuse=1, shared_grad=False, check_every=None):
+    """Runs both sides for `steps` updates; checks after the first update, at chosen steps and at the end."""
+    g = H.GpuRun(w, fuse=fuse, shared_grad=shared_grad)
+    o = H.OracleRun(w, slabs, shared_grad=shared_grad)
+    steps = steps or w.total_steps
+    worst = 0.0
+    try:
+        for i in range(steps):
+            perm = g.perm0()
+            assert perm == o.o.perm_lr[0]
+            ended = g.step(perm)
+            assert ended == o.step()
+            if i == 0:
+                worst = max(worst, H.compare_slabs(g, o, TOL_ONE_STEP))
+            elif check_every and (i + 1) % check_every == 0:
+                worst = max(worst, H.compare_slabs(g, o, TOL_FULL_RUN))
+            if ended or i == 0:
+                H.compare_scalars(g.state(), o.o, w.n_replicas, w.n_groups)
+        worst = max(worst, H.compare_slabs(g, o, TOL_FULL_RUN))
+        st = g.state()
+        assert st.device_status == 0
+        H.compare_scalars(st, o.o, w.n_replicas, w.n_groups)
+    finally:
+        g.close()
+    return worst
+
+
+def test_device_fill_matches_the_numpy_generator_bit_for_bit():
+    import torch
+    from hdet_inputs import device as D
+    key = G.stream_key(5, G.STREAM_GRAD, 7, 3)
+    n, start = 100003, 12345
+    for sigma in (1e-3, 0.02):
+        sc = G.scale_for_sigma(sigma)
+        a = torch.empty(n, dtype=torch.float32, device="cuda")
+        D.fill(a, key, start, sc)
+        assert np.array_equal(a.cpu().numpy().view(np.uint32), G.fill_f32(key, start, n, sc).view(np.uint32))
+        b = torch.empty(n, dtype=torch.bfloat16, device="cuda")
+        D.fill(b, key, start, sc)
+        assert np.array_equal(b.view(torch.int16).cpu().numpy().view(np.uint16), G.fill_bf16_bits(key, start, n, sc))
+
+
+def test_config1_sgd_every_element_every_step():
+    w = W.config1()
+    worst = _lockstep(w, H.whole_tensor_slabs(w), check_every=1)
+    assert worst <= TOL_FULL_RUN
+
+
+@pytest.mark.parametrize("optimizer,grad_dtype", [(W.OPT_ADAMW, W.DTYPE_BF16), (W.OPT_ADAMW, W.DTYPE_F32),
+                                                   (W.OPT_SGD, W.DTYPE_F32), (W.OPT_SGD, W.DTYPE_BF16)])
+@pytest.mark.parametrize("align", [8, 1])
+def test_ragged_list_every_element(optimizer, grad_dtype, align):
+    """Odd sizes: tails shorter than a vector, exact tile multiples, one element; align=1 forces scalar accesses."""
+    w = W.ragged_workload(n_replicas=3, optimizer=optimizer, grad_dtype=grad_dtype, align_elems=align)
+    _lockstep(w, H.whole_tensor_slabs(w), check_every=1)
+
+
+@pytest.mark.parametrize("n", [1, 2, 5, 32])
+def test_replica_counts(n):
+    w = W.ragged_workload(n_replicas=n, numels=(4099, 2048, 3))
+    _lockstep(w, H.whole_tensor_slabs(w), check_every=3)
+
+
+def test_shared_gradient_stride_zero():
+    w = W.ragged_workload(n_replicas=4, numels=(5000, 17, 2048))
+    _lockstep(w, H.whole_tensor_slabs(w), shared_grad=True, check_every=3)
+    w = replace(W.config1(), tensors=(W.TensorSpec("flat", 10007, 0),))
+    _lockstep(w, H.whole_tensor_slabs(w), shared_grad=True, check_every=4)
+
+
+def _final_arena(w, fuse=1, shared_grad=False, steps=None):
+    g = H.GpuRun(w, fuse=fuse, shared_grad=shared_grad)
+    for i in range(steps or w.total_steps):
+        g.step(g.perm0())
+    a = g.arena
+    out = [a.param.clone()] + ([a.exp_avg.clone(), a.exp_avg_sq.clone()] if a.exp_avg is not None else [])
+    launches = g.B.hdet_kernel_launches(g.h)
+    g.close()
+    return out, launches
+
+
+def test_fused_converge_equals_update_then_converge_bitwise_and_runs_are_deterministic():
+    import torch
+    w = W.ragged_workload(n_replicas=5, numels=(1, 7, 4097, 2048, 12289))
+    fused, l1 = _final_arena(w, fuse=1)
+    again, _ = _final_arena(w, fuse=1)
+    unfused, l2 = _final_arena(w, fuse=0)
+    for a, b, c in zip(fused, again, unfused):
+        assert torch.equal(a, b)
+        assert torch.equal(a, c)
+    assert l1 == w.total_steps and l2 == w.total_steps + w.total_steps // w.sync_interval
+
+
+def test_alpha_zero_keeps_replicas_bitwise_identical():
+    import torch
+    w = replace(W.ragged_workload(n_replicas=6, numels=(4097, 33)), alpha_lr=0.0, alpha_wd=0.0, autolr=0)
+    g = H.GpuRun(w, shared_grad=True)
+    for i in range(7):
+        g.step()
+        for t in (g.arena.param, g.arena.exp_avg, g.arena.exp_avg_sq):
+            assert torch.equal(t, t[0:1].expand_as(t))
+    g.close()
+
+
+def test_padding_between_tensors_is_never_written():
+    import torch
+    w = W.ragged_workload(n_replicas=3)
+    g = H.GpuRun(w)
+    mask = torch.ones(g.arena.p_pad, dtype=torch.bool, device="cuda")
+    for off, t in zip(g.arena.offsets, w.tensors):
+        mask[off:off + t.numel] = False
+    assert mask.any()
+    for i in range(w.total_steps):
+        g.step(g.perm0())
+    for t in (g.arena.param, g.arena.exp_avg, g.arena.exp_avg_sq):
+        assert torch.all(t[:, mask] == 0)
+    g.close()
+
+
+def test_standalone_converge_matches_oracle_mean():
+    import torch
+    from oracle import hdet_oracle as O
+    w = W.ragged_workload(n_replicas=7, numels=(4099, 5, 2048))
+    g = H.GpuRun(w)
+    torch.manual_seed(0)
+    g.arena.param.copy_(torch.randn_like(g.arena.param))
+    before = g.arena.param.cpu().numpy().astype(np.float64)
+    m0 = g.arena.exp_avg.clone()
+    g.B.hdet_converge(g.h)
+    after = g.arena.param.cpu().numpy()
+    for off, t in zip(g.arena.offsets, w.tensors):
+        ref = before[:, off:off + t.numel].copy()
+        O.converge(ref)
+        assert H.rel_err(after[:, off:off + t.numel], ref).max() <= 1e-7
+    assert torch.equal(g.arena.exp_avg, m0)
+    assert g.state().step == 0
+    g.close()
+
+
+def test_nonfinite_parameter_sets_the_status_word():
+    import torch
+    w = W.ragged_workload(n_replicas=2, numels=(3000,))
+    g = H.GpuRun(w)
+    g.step()
+    assert g.state().device_status == 0
+    g.arena.grad[1, 5] = float("inf")
+    g.B.hdet_step(g.h, None)
+    with pytest.raises(g.B.HdetError) as e:
+        g.B.hdet_get_state(g.h)
+    assert e.value.status == g.B.HDET_ERR_NONFINITE
+    st = g.B.hdet_get_state(g.h, raise_on_nonfinite=False)
+    assert st.device_status & 1
+    g.B.hdet_set_state(g.h, st)            # clears the word
+    assert g.B.hdet_get_state(g.h).device_status == 0
+    g.close()
+
+
+def test_config2_full_run_sampled():
+    """N=8, 25.19 M parameters, AdamW, one-cycle over 1000 updates, T=50, controller on: the full run."""
+    w = W.config2()
+    slabs = [(k, 0, min(2048, t.numel)) for k, t in enumerate(w.tensors)]
+    slabs += [(0, 2097152 - 4096, 4096), (10, 1024 * 1024 + 2048 * 7, 2048), (22, 2048 * 513, 2048)]
+    worst = _lockstep(w, slabs, check_every=250)
+    assert worst <= TOL_FULL_RUN
+
+
+def _decoder_sample(w, n_small=12, n_big=10, seed=0):
+    """First tile of some small tensors; first, last (ragged tail) and a random tile of some matrices."""
+    rng = np.random.default_rng(seed)
+    small = [k for k, t in enumerate(w.tensors) if t.numel <= 8192]
+    big = [k for k, t in enumerate(w.tensors) if t.numel > 8192]
+    slabs = [(int(k), 0, w.tensors[k].numel if w.tensors[k].numel <= 2048 else 2048)
+             for k in rng.choice(small, n_small, replace=False)]
+    picks = [0, 1, big[-1]] + [int(k) for k in rng.choice(big[2:-1], n_big - 3, replace=False)]
+    for k in picks:
+        n = w.tensors[k].numel
+        j = int(rng.integers(1, n // 2048 - 1))
+        slabs += [(k, 0, 2048), (k, n - 2048 - 1000, 2048 + 1000), (k, j * 2048, 2048)]
+    return slabs
+
+
+def _free_gb():
+    import torch
+    return torch.cuda.mem_get_info()[0] / 1e9
+
+
+def test_config3_full_size_sampled():
+    """N=8, 354.8 M parameters in 292 tensors (39.7 GB resident), 500 updates, T=100, controller on."""
+    w = W.config3()
+    if _free_gb() < 45:
+        pytest.skip("needs 45 GB of free device memory")
+    _lockstep(w, _decoder_sample(w, 10, 8), check_every=250)
+
+
+def test_config4_full_size_sampled():
+    """N=8, 1.316 B parameters (147.4 GB resident), T=1: every update is the fused update+converge kernel."""
+    w = W.config4()
+    if _free_gb() < 152:
+        pytest.skip("needs 152 GB of free device memory")
+    _lockstep(w, _decoder_sample(w, 12, 10), check_every=10)
+
+
+@pytest.mark.parametrize("T", [1, 10, 100])
+def test_config5_n16_weight_decay_spread(T):
+    """N=16, 124.4 M parameters, learning-rate and weight-decay spread, 300 updates, controller on."""
+    w = W.config5(T)
+    if _free_gb() < 32:
+        pytest.skip("needs 32 GB of free device memory")
+    _lockstep(w, _decoder_sample(w, 6, 5), check_every=100)
