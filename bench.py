@@ -1,0 +1,342 @@
+"""Benchmark of the HDET hot path on B200: fan-out update + converge + controller call, one step per launch.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload config4] [--impl ours|reference]
+
+A step is one pass of the whole hot path over the resident workload: hdet_step (spread and schedule
+scalars on the host, one fused fan-out update kernel; on the last update of a round the same kernel also
+forms the replica mean) followed by hdet_autolr_update when the step ended a round.  The default
+workload is the 1.3 B-parameter decoder list with N = 8 replicas and T = 1 (every step is the fused
+update+converge kernel, 147 GB resident); it falls back to the 350 M list when the device has less
+free memory.  Gradients are generated once on the device and held fixed during timing (147 GB of
+inputs is far larger than L2, so no flush is needed).  With --gpus N > 1 every rank runs an
+independent copy of the workload on its own GPU (the path has no inter-GPU exchange): weak scaling.
+
+Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+from hdet_inputs import recipes as R  # noqa: E402
+from hdet_inputs import workloads as W  # noqa: E402
+
+METRIC = "fan-out step+converge throughput (replica-parameter-elements updated per second)"
+UNIT = "replica-param-elements/s"
+FALLBACK_HBM_GBS = 6650.0
+NOMINAL_HBM_GBS = 8000.0
+
+
+def bytes_per_element(w: W.Workload) -> int:
+    """Algorithmic HBM bytes per replica-parameter-element of the fan-out kernel (fused converge adds none)."""
+    g = 2 if w.grad_dtype == W.DTYPE_BF16 else 4
+    if w.optimizer == W.OPT_ADAMW:
+        return 12 + g + 12           # read theta, m, v, g; write theta, m, v
+    return 4 + g + 4                 # read theta, g; write theta
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    return FALLBACK_HBM_GBS, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+def oracle_sample(w: W.Workload, n_slabs: int = 32, slab: int = 65536):
+    """Bounded sample of the workload for the CPU oracle: n_slabs ranges of `slab` elements from the largest tensors."""
+    big = sorted(range(len(w.tensors)), key=lambda k: -w.tensors[k].numel)
+    slabs = []
+    for j in range(n_slabs):
+        k = big[j % max(1, min(len(big), 8))]
+        n = min(slab, w.tensors[k].numel)
+        start = (j * 7919 * slab) % max(1, w.tensors[k].numel - n + 1)
+        slabs.append((k, start // 8 * 8, n))
+    return slabs
+
+
+class OracleBench:
+    """The CPU oracle, as it stands, on a bounded sample (numpy, one thread)."""
+
+    def __init__(self, w: W.Workload):
+        sys.path.insert(0, os.path.join(ROOT, "tests"))
+        import harness as H
+        self.w = w
+        self.slabs = oracle_sample(w)
+        self.run = H.OracleRun(w, self.slabs)
+        self.grads = self.run.grads(0)                      # held fixed, as on the GPU
+        self.units = sum(n for (_, _, n) in self.slabs) * w.n_replicas
+
+    def step(self):
+        self.run.o.step(self.grads, R.step_losses(self.w, self.run.o.i % self.w.total_steps, self.run.o.perm_lr[0]))
+
+    def describe(self):
+        return (f"{len(self.slabs)} ranges x {self.slabs[0][2]} elements x N={self.w.n_replicas} replicas of "
+                f"{self.w.name} ({self.units} replica-elements per step), gradients held fixed")
+
+
+def time_oracle(w, steps, warmup):
+    ob = OracleBench(w)
+    for _ in range(warmup):
+        ob.step()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        ob.step()
+    dt = time.perf_counter() - t0
+    return ob, ob.units * steps / dt, dt / steps
+
+
+class ClockSampler:
+    """nvidia-smi clock/throttle samples taken while the timed region runs."""
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.proc = None
+        self.gpu = gpu_index
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(gpu_index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            p = [x.strip() for x in line.split(",")]
+            if len(p) < 9:
+                continue
+            try:
+                sm.append(float(p[1])); mx.append(float(p[2]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, p[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        busy = sm[len(sm) // 4:] if len(sm) >= 4 else sm      # skip the ramp at the start
+        return {"sm_mhz": statistics.median(busy), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def pick_workload(name, torch, sync_interval=None):
+    w = W.ALL_CONFIGS[name]()
+    if sync_interval:
+        from dataclasses import replace
+        w = replace(w, sync_interval=sync_interval, name=f"{w.name}_T{sync_interval}")
+    need = w.n_replicas * w.arena_numel() * (bytes_per_element(w) - 12 if w.optimizer == W.OPT_ADAMW else 8)
+    free, _ = torch.cuda.mem_get_info()
+    note = None
+    if need + (3 << 30) > free:
+        note = f"{name} needs {need / 1e9:.1f} GB but only {free / 1e9:.1f} GB are free: fell back to config3"
+        w = W.config3()
+    return w, note
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    from hdet_inputs import device as D
+    from paper_2604_24708_b200 import binding as B
+    from paper_2604_24708_b200 import from_workload
+    from paper_2604_24708_b200.arena import StackedArena
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+
+    w, note = pick_workload(args.workload, torch, args.sync_interval)
+    n, P = w.n_replicas, w.numel
+    arena = StackedArena([t.numel for t in w.tensors], [t.group for t in w.tensors], n, w.optimizer, w.grad_dtype,
+                         device=f"cuda:{local}", align_elems=w.align_elems)
+    D.fill(arena.param[0], R.param_key(w), 0, R.param_scale(w))
+    for r in range(1, n):
+        arena.param[r].copy_(arena.param[0])
+    for r in range(n):
+        D.fill(arena.grad[r], R.grad_key(w, 0, r), 0, R.grad_scale(w))
+    h = B.hdet_create(from_workload.config_for(w, fuse=1, device=local), arena.descriptors())
+    B.hdet_set_schedule(h, from_workload.schedule_for(w))
+    stream = torch.cuda.current_stream()
+    losses = [list(R.step_losses(w, i % w.total_steps)) for i in range(w.total_steps)]
+    state = {"i": 0}
+
+    def one_step():
+        if B.hdet_step(h, losses[state["i"] % w.total_steps], stream.cuda_stream):
+            B.hdet_autolr_update(h)
+        state["i"] += 1
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        one_step()
+    barrier()
+
+    # ---- device-timed region: inputs resident in HBM -------------------------------------------------
+    sampler = ClockSampler(local) if rank == 0 else None
+    launches0 = B.hdet_kernel_launches(h)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    barrier()
+    ev[0].record(stream)
+    for k in range(args.steps):
+        one_step()
+        ev[k + 1].record(stream)
+    barrier()
+    clocks = sampler.stop() if sampler else None
+    launches = B.hdet_kernel_launches(h) - launches0
+    total_ms = ev[0].elapsed_time(ev[-1])
+    per_step_ms = [ev[k].elapsed_time(ev[k + 1]) for k in range(args.steps)]
+    t = torch.tensor([total_ms], dtype=torch.float64, device=f"cuda:{local}")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms_max = float(t.item())
+    ms_per_step = total_ms_max / args.steps
+    units_per_step = n * P * world
+    value = units_per_step / (ms_per_step * 1e-3)
+
+    # ---- end-to-end region: this step's gradients come from pinned host memory, the status word goes back --
+    e2e_steps = max(1, min(args.steps, args.e2e_steps))
+    host_grad = torch.empty(arena.p_pad, dtype=arena.grad.dtype).pin_memory()
+    host_grad.copy_(arena.grad[0].cpu())
+    h2d_bytes = n * arena.p_pad * arena.grad.element_size()
+
+    def e2e_step():
+        for r in range(n):
+            arena.grad[r].copy_(host_grad, non_blocking=True)
+        one_step()
+        st = B.hdet_get_state(h, raise_on_nonfinite=False)   # reads the device status word back (synchronises)
+        return st.device_status
+
+    e2e_step()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record(stream)
+    barrier()
+    t2 = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=f"cuda:{local}")
+    if world > 1:
+        dist.all_reduce(t2, op=dist.ReduceOp.MAX)
+    e2e_value = units_per_step * e2e_steps / (float(t2.item()) * 1e-3)
+    final_state = B.hdet_get_state(h, raise_on_nonfinite=False)
+    B.hdet_destroy(h)
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    bpe = bytes_per_element(w)
+    peak, peak_src = measured_peaks()
+    launch_ms = statistics.mean(per_step_ms) / max(1, launches // args.steps)
+    achieved = bpe * n * P / (launch_ms * 1e-3) / 1e9
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32 (bf16 gradients, fp64 replica sum)" if w.grad_dtype == W.DTYPE_BF16 else "f32",
+        "data": "synthetic (seeded integer generator; gradients held fixed during timing)",
+        "config": {
+            "workload": w.name, "n_replicas": n, "params_per_replica": P, "n_tensors": len(w.tensors),
+            "optimizer": "adamw" if w.optimizer == W.OPT_ADAMW else "sgd", "sync_interval": w.sync_interval,
+            "alpha_lr": w.alpha_lr, "resident_gb": arena.resident_bytes() / 1e9,
+            "l2_policy": "inputs larger than L2 (no flush)", "parallelism": f"{world} independent replicas of the job",
+            "note": note,
+        },
+        "param_elements_per_s": value / n,
+        "hbm_frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d_bytes, "d2h_bytes_per_step": 4,
+                "steps": e2e_steps,
+                "what": "per step: gradients of all replicas copied from pinned host memory, hdet_step "
+                        "(+ hdet_autolr_update), device status word read back"},
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "traffic": args.traffic_bytes, "peak_source": peak_src,
+                     "kernel": "fanout_kernel (fused update+converge)" if w.sync_interval == 1 else "fanout_kernel",
+                     "bytes_per_element": bpe, "launch_ms": launch_ms},
+        "device_status": int(final_state.device_status),
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        ob, v, sec = time_oracle(w, args.cpu_steps, 1)
+        out["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": ob.describe(),
+                               "s_per_step": sec, "steps": args.cpu_steps}
+    print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def run_reference(args):
+    """The reference arm: the CPU oracle, as it stands, on a bounded sample per step (rank 0 only)."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    w = W.ALL_CONFIGS[args.workload]()
+    ob, v, sec = time_oracle(w, args.steps, max(args.warmup, 1))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    out = {
+        "impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 1), "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic (seeded integer generator)",
+        "config": {"workload": w.name, "n_replicas": w.n_replicas, "params_per_replica": w.numel,
+                   "sample": ob.describe()},
+        "cpu_baseline": {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": ob.describe()},
+        "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(out))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="config4", choices=sorted(W.ALL_CONFIGS))
+    ap.add_argument("--sync-interval", type=int, default=None,
+                    help="override the workload's T (e.g. 1 to profile the fused update+converge kernel on a small list)")
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--cpu-steps", type=int, default=30)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--traffic-bytes", type=float, default=None,
+                    help="dram bytes per launch of the dominant kernel from an ncu capture (reported as roofline.traffic)")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

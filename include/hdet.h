@@ -162,6 +162,7 @@ HDET_API int hdet_create(const hdet_config* cfg, const hdet_tensor* tensors, int
  * list (one-cycle policy with cosine or linear annealing, or a constant) and the
  * controller constants (beta, sigma, lambda of Eq. 4 / Eq. 7; f_div, f_final of Eq. 8;
  * S_warm).  May be called again at any time; it does not reset the step count.
+ * Updates past step S keep the rate of step S - 1.
  * Errors: INVALID_ARG (NULL, S < 1, max_lr NULL, p*S <= 1 or p >= 1 for a one-cycle
  * kind, factors <= 0, sigma <= 0 with autolr, f_div or f_final <= 0).
  */

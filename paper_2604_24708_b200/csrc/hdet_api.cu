@@ -271,12 +271,10 @@ int hdet_step(hdet_handle h, const double* step_losses, void* stream, int32_t* d
     }
     for (int g = 0; g < G; ++g)
       for (int r = 0; r < n; ++r) {
-        s.decay[g][r] = adam ? (float)(1.0 - h->lr[g][r] * h->wd[g][r]) : 1.0f;
+        s.lr_wd[g][r] = adam ? (float)(h->lr[g][r] * h->wd[g][r]) : 0.0f;
         s.step[g][r] = (float)(adam ? h->lr[g][r] / bc1 : h->lr[g][r]);
       }
-    s.beta1 = (float)h->cfg.beta1;
     s.one_minus_beta1 = (float)(1.0 - h->cfg.beta1);
-    s.beta2 = (float)h->cfg.beta2;
     s.one_minus_beta2 = (float)(1.0 - h->cfg.beta2);
     s.rsqrt_bc2 = (float)(1.0 / std::sqrt(bc2));
     s.eps = (float)h->cfg.eps;

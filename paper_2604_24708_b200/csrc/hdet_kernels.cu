@@ -16,19 +16,22 @@ namespace hdet {
 namespace {
 
 struct AdamConsts {
-  float beta1, one_minus_beta1, beta2, one_minus_beta2, rsqrt_bc2, eps;
+  float one_minus_beta1, one_minus_beta2, rsqrt_bc2, eps;
 };
 
 // Adam with decoupled weight decay on one element (Section 4.1 names Adam; weight decay is a
 // spreadable scalar per Remark 1):
 //   theta *= 1 - lr*wd ; m = b1 m + (1-b1) g ; v = b2 v + (1-b2) g^2 ;
 //   theta -= lr/(1-b1^t) * m / (sqrt(v)/sqrt(1-b2^t) + eps)
-__device__ __forceinline__ void adam_element(float& th, float& m, float& v, float g, float decay, float step,
+// The moving averages are evaluated as x + (1-b)(new - x) and the decay as theta - (lr*wd) theta:
+// the fp32 images of b2 = 0.999 and of 1 - lr*wd are off by ~1e-8 relative, which the recurrences
+// would amplify to ~1e-5 over a thousand updates; the small factors 1-b and lr*wd carry no such bias.
+__device__ __forceinline__ void adam_element(float& th, float& m, float& v, float g, float lr_wd, float step,
                                              const AdamConsts& c) {
-  m = fmaf(c.beta1, m, c.one_minus_beta1 * g);
-  v = fmaf(c.beta2, v, c.one_minus_beta2 * g * g);
+  m = fmaf(c.one_minus_beta1, g - m, m);
+  v = fmaf(c.one_minus_beta2, fmaf(g, g, -v), v);
   const float denom = fmaf(sqrtf(v), c.rsqrt_bc2, c.eps);
-  th = fmaf(-step, m / denom, th * decay);
+  th = fmaf(-step, m / denom, fmaf(-lr_wd, th, th));
 }
 
 // Eq. 2: theta <- theta - eta_r * g
@@ -69,7 +72,7 @@ __device__ void range_scalar(const TensorDesc& td, long long begin, long long en
       if (kAdam) {
         float m = __ldcs(td.exp_avg + r * td.state_stride + e);
         float v = __ldcs(td.exp_avg_sq + r * td.state_stride + e);
-        adam_element(th, m, v, g, s.decay[td.group][r], s.step[td.group][r], c);
+        adam_element(th, m, v, g, s.lr_wd[td.group][r], s.step[td.group][r], c);
         __stcs(td.exp_avg + r * td.state_stride + e, m);
         __stcs(td.exp_avg_sq + r * td.state_stride + e, v);
       } else {
@@ -144,7 +147,7 @@ __device__ __forceinline__ void tile_vector(const TensorDesc& td, long long off,
   }
 
   auto update_store = [&](Regs& b, int r) {
-    const float decay = s.decay[grp][r];
+    const float lr_wd = s.lr_wd[grp][r];
     const float step = s.step[grp][r];
 #pragma unroll
     for (int k = 0; k < kTileVecs; ++k) {
@@ -155,7 +158,7 @@ __device__ __forceinline__ void tile_vector(const TensorDesc& td, long long off,
         float m[4] = {b.m[k].x, b.m[k].y, b.m[k].z, b.m[k].w};
         float v[4] = {b.v[k].x, b.v[k].y, b.v[k].z, b.v[k].w};
 #pragma unroll
-        for (int q = 0; q < 4; ++q) adam_element(th[q], m[q], v[q], g[q], decay, step, c);
+        for (int q = 0; q < 4; ++q) adam_element(th[q], m[q], v[q], g[q], lr_wd, step, c);
         if (ok[k]) {
           __stcs(reinterpret_cast<float4*>(M + r * ss + idx[k]), make_float4(m[0], m[1], m[2], m[3]));
           __stcs(reinterpret_cast<float4*>(V + r * ss + idx[k]), make_float4(v[0], v[1], v[2], v[3]));
@@ -202,7 +205,7 @@ __device__ __forceinline__ void tile_vector(const TensorDesc& td, long long off,
 template <typename GradT, bool kAdam, bool kConv>
 __global__ void __launch_bounds__(kThreads, 2)
 fanout_kernel(const __grid_constant__ LaunchPlan plan, const __grid_constant__ StepScalars s) {
-  const AdamConsts c{s.beta1, s.one_minus_beta1, s.beta2, s.one_minus_beta2, s.rsqrt_bc2, s.eps};
+  const AdamConsts c{s.one_minus_beta1, s.one_minus_beta2, s.rsqrt_bc2, s.eps};
   bool bad = false;
   for (int t = blockIdx.x; t < plan.n_tiles; t += gridDim.x) {
     const Tile tile = plan.tiles[t];

@@ -35,9 +35,9 @@ struct Tile {
 
 // Per-launch scalars, passed by value as kernel parameters (no device table to update).
 struct StepScalars {
-  float decay[HDET_MAX_GROUPS][HDET_MAX_REPLICAS];  // 1 - lr*wd
+  float lr_wd[HDET_MAX_GROUPS][HDET_MAX_REPLICAS];  // lr * wd (decoupled decay factor is 1 - lr_wd)
   float step[HDET_MAX_GROUPS][HDET_MAX_REPLICAS];   // AdamW: lr / (1 - beta1^t); SGD: lr
-  float beta1, one_minus_beta1, beta2, one_minus_beta2;
+  float one_minus_beta1, one_minus_beta2;
   float rsqrt_bc2;  // 1 / sqrt(1 - beta2^t)
   float eps;
   double inv_n;     // 1 / N

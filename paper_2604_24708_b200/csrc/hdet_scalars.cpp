@@ -20,7 +20,7 @@ double base_rate(int kind, int64_t i, int64_t total_steps, double max_lr, double
   const double floor_lr = lo / final_div_factor;
   const double knee = pct_start * (double)total_steps - 1.0;
   const double last = (double)total_steps - 1.0;
-  const double x = (double)i;
+  const double x = std::min((double)i, last);  // past the last scheduled step the final rate is held
   double from, to, frac;
   if (x <= knee) {
     from = lo; to = max_lr; frac = x / knee;

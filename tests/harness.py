@@ -12,18 +12,13 @@ from oracle import hdet_oracle as O
 
 # ----------------------------------------------------------------------------- library side
 def lib_config(B, w: W.Workload, fuse: int = 1, device: int = 0):
-    return B.hdet_config(
-        n_replicas=w.n_replicas, n_groups=w.n_groups, optimizer=w.optimizer, grad_dtype=w.grad_dtype,
-        beta1=w.beta1, beta2=w.beta2, eps=w.eps, momentum=0.0, alpha_lr=w.alpha_lr, alpha_wd=w.alpha_wd,
-        sync_interval=w.sync_interval, reshuffle=w.reshuffle, fuse_converge=fuse, seed=w.seed, device=device)
+    from paper_2604_24708_b200 import from_workload
+    return from_workload.config_for(w, fuse, device)
 
 
 def lib_schedule(B, w: W.Workload):
-    return B.make_schedule(
-        w.sched_kind, w.total_steps, list(w.max_lr), list(w.weight_decay), pct_start=w.pct_start,
-        div_factor=w.div_factor, final_div_factor=w.final_div_factor, autolr=w.autolr,
-        warmup_steps=w.warmup_steps, beta=w.ctrl_beta, sigma=w.ctrl_sigma, lambda_=w.ctrl_lambda,
-        f_div=w.f_div, f_final=w.f_final)
+    from paper_2604_24708_b200 import from_workload
+    return from_workload.schedule_for(w)
 
 
 class GpuRun:
@@ -82,6 +77,8 @@ class GpuRun:
         self.torch.cuda.synchronize()
         self.B.hdet_destroy(self.h)
         self.h = None
+        self.arena = None
+        self.torch.cuda.empty_cache()
 
 
 # ----------------------------------------------------------------------------- oracle side
