@@ -224,8 +224,39 @@ HDET_API int hdet_set_state(hdet_handle h, const hdet_state* in);
 /* hdet_destroy -- frees the work table and the handle.  NULL is accepted. */
 HDET_API int hdet_destroy(hdet_handle h);
 
-/* hdet_last_error -- text of the last failure on h (or of the last failed hdet_create
- * when h is NULL).  The pointer stays valid until the next call on that handle. */
+/*
+ * hdet_converge_static -- (the paper has no counterpart: this is a packaging variant of
+ * hdet_converge.)  Averages the N replicas of every listed tensor like hdet_converge, but needs
+ * no handle and never allocates device memory.  It is meant for callers that cannot call
+ * cudaMalloc at the point where they need the mean: code running under a framework that has
+ * handed all device memory to its own pool, or a latency-critical loop where an allocation
+ * (which may synchronise the device) is not acceptable.
+ *
+ * The caller passes the same hdet_tensor descriptors as to hdet_create; only param, numel and
+ * param_stride are read (grad and the moments may be NULL).  The work tables that hdet_create
+ * would put in allocated memory are written, on every call, into one static device array of
+ * about 0.6 MB that each GPU loading the library holds until the process exits.  Limits, checked
+ * before anything is launched: at most HDET_STATIC_MAX_TENSORS tensors and HDET_STATIC_MAX_TILES
+ * tiles of 2048 elements in total (each tensor occupies ceil(numel / 2048) tiles, so at most
+ * 134,217,728 elements per replica); larger lists return HDET_ERR_UNSUPPORTED with a message and
+ * should use hdet_converge.
+ *
+ * The first call on a device resolves the array's device address (cudaGetSymbolAddress) and
+ * queries the launch shape; make that first call outside any stream capture.  All calls share the
+ * array, which keeps the previous call's contents: each call clears the status word and rewrites
+ * the tables it uses, in stream order.  Two calls whose work overlaps on the GPU (different
+ * streams without an event between them, or different host threads) race on the array and must
+ * be serialised by the caller.  The copies of the tables come from pageable host memory, so the
+ * call may wait for earlier work on `stream`.
+ * Errors: INVALID_ARG, ALIGN, UNSUPPORTED (limits), CUDA; text via hdet_last_error(NULL).
+ */
+#define HDET_STATIC_MAX_TENSORS 1024
+#define HDET_STATIC_MAX_TILES 65536
+HDET_API int hdet_converge_static(const hdet_tensor* tensors, int64_t n_tensors, int32_t n_replicas,
+                                  int32_t device, void* stream);
+
+/* hdet_last_error -- text of the last failure on h (when h is NULL: of the last failed call
+ * that has no handle, hdet_create or hdet_converge_static, on this thread).  The pointer stays valid until the next call on that handle. */
 HDET_API const char* hdet_last_error(hdet_handle h);
 
 /* hdet_kernel_launches -- number of kernels this handle has launched so far. */

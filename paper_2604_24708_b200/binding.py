@@ -97,6 +97,8 @@ def _load() -> C.CDLL:
     lib.hdet_last_error.restype = C.c_char_p
     lib.hdet_kernel_launches.argtypes = [H]
     lib.hdet_kernel_launches.restype = C.c_int64
+    lib.hdet_converge_static.argtypes = [C.POINTER(hdet_tensor), C.c_int64, C.c_int32, C.c_int32, C.c_void_p]
+    lib.hdet_converge_static.restype = C.c_int
     for f in ("hdet_create", "hdet_set_schedule", "hdet_step", "hdet_converge", "hdet_autolr_update",
               "hdet_get_state", "hdet_set_state", "hdet_destroy"):
         getattr(lib, f).restype = C.c_int
@@ -184,6 +186,21 @@ def hdet_step(h, step_losses: Optional[Sequence[float]] = None, stream: int = 0)
 
 def hdet_converge(h, stream: int = 0) -> None:
     _check(_lib.hdet_converge(h, C.c_void_p(stream)), h)
+
+
+HDET_STATIC_MAX_TENSORS = 1024
+HDET_STATIC_MAX_TILES = 65536
+
+
+def hdet_converge_static(tensors: Sequence[hdet_tensor], n_replicas: int, device: int = 0, stream: int = 0) -> None:
+    """Replica mean of every listed tensor without a handle and without any device allocation.
+
+    For callers that cannot allocate at that point (all device memory owned by a framework pool, or a
+    loop that must not risk the synchronisation an allocation can cause).  The work tables go into a
+    static device array shared by all calls, so calls that overlap on the GPU must be serialised.
+    """
+    arr = (hdet_tensor * len(tensors))(*tensors) if tensors else None
+    _check(_lib.hdet_converge_static(arr, len(tensors), n_replicas, device, C.c_void_p(stream)), None)
 
 
 def hdet_autolr_update(h, round_losses: Optional[Sequence[float]] = None, stream: int = 0) -> None:

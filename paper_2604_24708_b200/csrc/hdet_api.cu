@@ -7,6 +7,7 @@
 #include <string>
 #include <vector>
 
+#include "hdet_internal.h"
 #include "hdet_kernels.cuh"
 #include "hdet_scalars.h"
 
@@ -111,6 +112,10 @@ bool is_permutation(const int32_t* p, int n) {
 }
 
 }  // namespace
+
+namespace hdet {
+void set_handleless_error(const char* msg) { g_create_error = msg ? msg : ""; }
+}  // namespace hdet
 
 extern "C" {
 
