@@ -34,6 +34,10 @@ from hdet_inputs import workloads as W  # noqa: E402
 
 METRIC = "fan-out step+converge throughput (replica-parameter-elements updated per second)"
 UNIT = "replica-param-elements/s"
+# DRAM bytes per replica-element of fanout_kernel<bf16, AdamW, converge>, from the ncu capture summarised in
+# profiles/fanout_adamw_bf16_converge__config2_T1_ncu_full.md (5.1830 GB over 8 x 25,190,400 elements); traffic grows
+# in proportion to N x P.  Set to None whenever that kernel changes until the counters are taken again.
+NCU_DRAM_BYTES_PER_ELEMENT_ADAMW_BF16_CONVERGE = 5.1830e9 / (8 * 25_190_400)
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
 
@@ -262,6 +266,11 @@ def run_ours(args):
     peak, peak_src = measured_peaks()
     launch_ms = statistics.mean(per_step_ms) / max(1, launches // args.steps)
     achieved = bpe * n * P / (launch_ms * 1e-3) / 1e9
+    traffic, traffic_src = args.traffic_bytes, "command line" if args.traffic_bytes else None
+    if (traffic is None and NCU_DRAM_BYTES_PER_ELEMENT_ADAMW_BF16_CONVERGE and w.optimizer == W.OPT_ADAMW
+            and w.grad_dtype == W.DTYPE_BF16 and w.sync_interval == 1):
+        traffic = NCU_DRAM_BYTES_PER_ELEMENT_ADAMW_BF16_CONVERGE * n * P
+        traffic_src = "ncu dram__bytes_read+write on the 25 M list, scaled by N*P (see profiles/)"
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
@@ -283,7 +292,7 @@ def run_ours(args):
                 "what": "per step: gradients of all replicas copied from pinned host memory, hdet_step "
                         "(+ hdet_autolr_update), device status word read back"},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": args.traffic_bytes, "peak_source": peak_src,
+                     "traffic": traffic, "traffic_source": traffic_src, "peak_source": peak_src,
                      "kernel": "fanout_kernel (fused update+converge)" if w.sync_interval == 1 else "fanout_kernel",
                      "bytes_per_element": bpe, "launch_ms": launch_ms},
         "device_status": int(final_state.device_status),

@@ -264,17 +264,6 @@ cudaError_t launch_one(const LaunchPlan& plan, const StepScalars& s, cudaStream_
   return cudaGetLastError();
 }
 
-template <typename GradT, bool kAdam>
-cudaError_t occupancy_one(int* out) {
-  int a = 0, b = 0;
-  cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&a, fanout_kernel<GradT, kAdam, false>, kThreads, 0);
-  if (e != cudaSuccess) return e;
-  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, fanout_kernel<GradT, kAdam, true>, kThreads, 0);
-  if (e != cudaSuccess) return e;
-  *out = a < b ? a : b;
-  return cudaSuccess;
-}
-
 }  // namespace
 
 cudaError_t launch_fanout(int optimizer, int grad_dtype, bool converge, const LaunchPlan& plan,
@@ -296,17 +285,6 @@ cudaError_t launch_converge(const LaunchPlan& plan, int n_replicas, cudaStream_t
   if (plan.n_tiles == 0) return cudaSuccess;
   converge_kernel<<<plan.grid, kThreads, 0, stream>>>(plan, n_replicas, 1.0 / (double)n_replicas);
   return cudaGetLastError();
-}
-
-cudaError_t fanout_occupancy(int optimizer, int grad_dtype, int* ctas_per_sm) {
-  const bool adam = optimizer == HDET_OPT_ADAMW;
-  const bool bf16 = grad_dtype == HDET_DTYPE_BF16;
-  if (adam) return bf16 ? occupancy_one<__nv_bfloat16, true>(ctas_per_sm) : occupancy_one<float, true>(ctas_per_sm);
-  return bf16 ? occupancy_one<__nv_bfloat16, false>(ctas_per_sm) : occupancy_one<float, false>(ctas_per_sm);
-}
-
-cudaError_t converge_occupancy(int* ctas_per_sm) {
-  return cudaOccupancyMaxActiveBlocksPerMultiprocessor(ctas_per_sm, converge_kernel, kThreads, 0);
 }
 
 }  // namespace hdet

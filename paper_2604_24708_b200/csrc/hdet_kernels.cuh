@@ -48,7 +48,7 @@ struct LaunchPlan {
   const TensorDesc* tensors;
   const Tile* tiles;
   int n_tiles;
-  int grid;            // CTAs to launch (persistent, grid-stride over tiles)
+  int grid;            // CTAs to launch; each takes tiles blockIdx.x, blockIdx.x + grid, ...
   unsigned* status;    // device status word; bit 0 = non-finite parameter seen
 };
 
@@ -59,9 +59,5 @@ cudaError_t launch_fanout(int optimizer, int grad_dtype, bool converge, const La
 
 // Stand-alone Eq. 3.
 cudaError_t launch_converge(const LaunchPlan& plan, int n_replicas, cudaStream_t stream);
-
-// Resident CTAs per SM of the fan-out kernels (minimum over the variants of one optimizer/dtype).
-cudaError_t fanout_occupancy(int optimizer, int grad_dtype, int* ctas_per_sm);
-cudaError_t converge_occupancy(int* ctas_per_sm);
 
 }  // namespace hdet
