@@ -146,6 +146,22 @@ class ClockSampler:
                 "samples": len(sm)}
 
 
+def max_over_ranks(ms: float, world: int, device="cpu") -> float:
+    """The slowest rank's time: every multi-GPU number is the max over ranks, never a mean or a wall clock."""
+    if world == 1:
+        return float(ms)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(units_per_rank: float, world: int, ms_per_step: float) -> float:
+    """Units all ranks processed per second (each rank runs its own copy of the job: weak scaling)."""
+    return units_per_rank * world / (ms_per_step * 1e-3)
+
+
 def pick_workload(name, torch, sync_interval=None):
     w = W.ALL_CONFIGS[name]()
     if sync_interval:
@@ -221,13 +237,8 @@ def run_ours(args):
     launches = B.hdet_kernel_launches(h) - launches0
     total_ms = ev[0].elapsed_time(ev[-1])
     per_step_ms = [ev[k].elapsed_time(ev[k + 1]) for k in range(args.steps)]
-    t = torch.tensor([total_ms], dtype=torch.float64, device=f"cuda:{local}")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms_max = float(t.item())
-    ms_per_step = total_ms_max / args.steps
-    units_per_step = n * P * world
-    value = units_per_step / (ms_per_step * 1e-3)
+    ms_per_step = max_over_ranks(total_ms, world, f"cuda:{local}") / args.steps
+    value = whole_job_value(n * P, world, ms_per_step)
 
     # ---- end-to-end region: this step's gradients come from pinned host memory, the status word goes back --
     e2e_steps = max(1, min(args.steps, args.e2e_steps))
@@ -250,10 +261,8 @@ def run_ours(args):
         e2e_step()
     e1.record(stream)
     barrier()
-    t2 = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=f"cuda:{local}")
-    if world > 1:
-        dist.all_reduce(t2, op=dist.ReduceOp.MAX)
-    e2e_value = units_per_step * e2e_steps / (float(t2.item()) * 1e-3)
+    e2e_ms = max_over_ranks(e0.elapsed_time(e1), world, f"cuda:{local}")
+    e2e_value = whole_job_value(n * P, world, e2e_ms / e2e_steps)
     final_state = B.hdet_get_state(h, raise_on_nonfinite=False)
     B.hdet_destroy(h)
 

@@ -475,6 +475,11 @@ def test_alg1_permutations_only_after_firing_and_independent_per_channel():
         assert lr[g].mean() == pytest.approx(base[g], rel=1e-14)                  # mean of the spread = base
         assert wd[g].mean() == pytest.approx(o.weight_decay[g], rel=1e-14, abs=1e-20)
         assert lr[g][0] == pytest.approx(base[g] * rho[o.perm_lr[g][0]], rel=1e-14)
+        # multipliers grow with their index, so each table is ordered like ITS OWN permutation
+        assert list(np.argsort(lr[g])) == list(np.argsort(o.perm_lr[g]))
+        if o.weight_decay[g] > 0:
+            assert list(np.argsort(wd[g])) == list(np.argsort(o.perm_wd[g]))
+            assert sorted(wd[g] / o.weight_decay[g]) == pytest.approx(sorted(O.spread_multipliers(n, 0.5)), rel=1e-13)
     assert np.all(wd[1] == 0.0)
 
 
@@ -505,3 +510,16 @@ def test_alg1_per_replica_rates_match_per_replica_library_runs():
             p.grad = torch.tensor(grads[i][r])
             opt.step()
         assert np.allclose(o.theta[0][r], p.detach().numpy(), rtol=1e-12, atol=1e-18)
+
+
+def test_alg1_controller_is_homogeneous_per_group():
+    """Eq. 5 - Eq. 7 are linear in the rates: a group whose rates are doubled gets twice Delta, v and eta_bar."""
+    n = 4
+    o = _mk(n, [2, 2], [0, 1], 2, sync_interval=3, total_steps=30, autolr=True, warmup_steps=3, reshuffle=False,
+            max_lr=[3e-4, 6e-4], weight_decay=[0.0, 0.0])
+    for i in range(9):
+        o.step([np.zeros(2)] * 2, 3.0 - 0.1 * np.linspace(-1, 1, n) + 0.01 * i)
+    assert o.fired and o.delta[0] > 0
+    assert o.delta[1] == pytest.approx(2 * o.delta[0], rel=1e-12)
+    assert o.vel[1] == pytest.approx(2 * o.vel[0], rel=1e-12)
+    assert o.ctrl_base[1] == pytest.approx(2 * o.ctrl_base[0], rel=1e-12)
