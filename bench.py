@@ -266,6 +266,36 @@ def run_ours(args):
     final_state = B.hdet_get_state(h, raise_on_nonfinite=False)
     B.hdet_destroy(h)
 
+    # ---- each kernel of the path on its own (same arena, a few launches each, after the headline timing) ----
+    per_kernel = {}
+    if not args.no_per_kernel:
+        from dataclasses import replace as _replace
+
+        def timed(fn, reps=5):
+            fn()
+            torch.cuda.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            for _ in range(reps):
+                fn()
+            b.record(stream)
+            torch.cuda.synchronize()
+            return a.elapsed_time(b) / reps
+
+        bpe_step = bytes_per_element(w)
+        for label, T, fuse, bpe_k in (("fanout_update", 1 << 40, 1, bpe_step),
+                                      ("fanout_update_converge_fused", 1, 1, bpe_step),
+                                      ("fanout_update_then_converge_unfused", 1, 0, bpe_step + 8)):
+            wk = _replace(w, sync_interval=T, autolr=0)
+            hk = B.hdet_create(from_workload.config_for(wk, fuse=fuse, device=local), arena.descriptors())
+            B.hdet_set_schedule(hk, from_workload.schedule_for(wk))
+            ms = timed(lambda: B.hdet_step(hk, None, stream.cuda_stream))
+            per_kernel[label] = {"ms": ms, "GB_per_s": bpe_k * n * P / ms / 1e6, "bytes_per_element": bpe_k}
+            if label == "fanout_update":
+                ms = timed(lambda: B.hdet_converge(hk, stream.cuda_stream))
+                per_kernel["converge_standalone"] = {"ms": ms, "GB_per_s": 8 * n * P / ms / 1e6, "bytes_per_element": 8}
+            B.hdet_destroy(hk)
+
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -304,6 +334,7 @@ def run_ours(args):
                      "traffic": traffic, "traffic_source": traffic_src, "peak_source": peak_src,
                      "kernel": "fanout_kernel (fused update+converge)" if w.sync_interval == 1 else "fanout_kernel",
                      "bytes_per_element": bpe, "launch_ms": launch_ms},
+        "per_kernel": per_kernel,
         "device_status": int(final_state.device_status),
     }
     if world == 1 and not args.no_cpu_baseline:
@@ -347,6 +378,7 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-steps", type=int, default=30)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-per-kernel", action="store_true", help="skip the per-kernel timings that follow the headline run")
     ap.add_argument("--traffic-bytes", type=float, default=None,
                     help="dram bytes per launch of the dominant kernel from an ncu capture (reported as roofline.traffic)")
     args = ap.parse_args()

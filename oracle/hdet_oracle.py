@@ -211,7 +211,9 @@ class HdetOracle:
 
     * update number t uses the schedule value at 0-based index t - 1; converge
       follows update t when t mod T = 0; "t >= S_warm" counts completed updates;
-    * gradients may differ per replica (general case) or be shared (Eq. 2);
+    * gradients may differ per replica (general case) or be shared (Eq. 2); with
+      grad_mean the per-replica gradients are first averaged over the replicas
+      (Algorithm 1, "AllReduce gradients") and every replica steps with that mean;
     * Adam moments are not averaged at converge (Eq. 3 averages "model
       parameters");
     * L_r is the mean loss over the last round (Section 3.4), so the accumulator
@@ -236,7 +238,7 @@ class HdetOracle:
                  ctrl_beta: float = 0.9, ctrl_sigma: float = 0.1, ctrl_lambda: float = 0.5,
                  f_div: float = 25.0, f_final: float = 1.0, reshuffle: bool = True, seed: int = 0,
                  beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8,
-                 n_replicas: Optional[int] = None):
+                 n_replicas: Optional[int] = None, grad_mean: bool = False):
         self.theta = [np.array(p, dtype=np.float64, copy=True) for p in params]
         self.n = self.theta[0].shape[0] if self.theta else int(n_replicas)
         self.m = [np.zeros_like(p) for p in self.theta]
@@ -256,6 +258,7 @@ class HdetOracle:
         self.f_div, self.f_final = f_div, f_final
         self.reshuffle, self.seed = bool(reshuffle), seed
         self.beta1, self.beta2, self.eps = beta1, beta2, eps
+        self.grad_mean = bool(grad_mean)
         # Algorithm 1, Init
         self.i = 0
         self.fired = False
@@ -304,6 +307,11 @@ class HdetOracle:
         for k, th in enumerate(self.theta):
             g_id = self.groups[k]
             gk = np.asarray(grads[k], dtype=np.float64)
+            if self.grad_mean and gk.ndim == 2:
+                g_bar = np.zeros(gk.shape[1], dtype=np.float64)     # Algorithm 1: AllReduce gradients (mean)
+                for r in range(n):
+                    g_bar += gk[r]
+                gk = g_bar / n
             for r in range(n):
                 g_r = gk if gk.ndim == 1 else gk[r]
                 if self.optimizer == SGD:

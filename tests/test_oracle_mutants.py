@@ -76,6 +76,8 @@ MUTANTS = [
     ("        for th in self.theta:\n            converge(th)", "        for th in self.theta + self.m:\n            converge(th)"),
     ("base[g] = self.ctrl_base[g] ", "base[g] = base_lr(self.sched_kind, self.i, self.S, self.ctrl_base[g], self.pct_start, self.div_factor, self.final_div_factor) "),
     ("sgd_update(th[r], g_r, lr[g_id][r])", "sgd_update(th[r], g_r, base[g_id])"),
+    ("gk = g_bar / n", "gk = g_bar"),
+    ("if self.grad_mean and gk.ndim == 2:", "if False:"),
     ("lr[g_id][r], wd[g_id][r],", "lr[g_id][r], self.weight_decay[g_id],"),
 ]
 

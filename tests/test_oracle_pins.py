@@ -523,3 +523,20 @@ def test_alg1_controller_is_homogeneous_per_group():
     assert o.delta[1] == pytest.approx(2 * o.delta[0], rel=1e-12)
     assert o.vel[1] == pytest.approx(2 * o.vel[0], rel=1e-12)
     assert o.ctrl_base[1] == pytest.approx(2 * o.ctrl_base[0], rel=1e-12)
+
+
+def test_alg1_gradient_mean_equals_a_run_with_the_mean_given_as_shared_gradient():
+    """Algorithm 1's gradient AllReduce: stepping with grad_mean on g_r is stepping on the shared mean of the g_r."""
+    rng = np.random.default_rng(12)
+    n = 5
+    a = _mk(n, [13, 4], [0, 0], 1, sync_interval=3, grad_mean=True)
+    b = _mk(n, [13, 4], [0, 0], 1, sync_interval=3)
+    for i in range(7):
+        gs = [rng.normal(scale=1e-3, size=(n, 13)), rng.normal(scale=1e-3, size=(n, 4))]
+        a.step(gs)
+        b.step([np.array([sum(g[r][j] for r in range(n)) / n for j in range(g.shape[1])]) for g in gs])
+        for k in range(2):
+            assert np.allclose(a.theta[k], b.theta[k], rtol=1e-13, atol=1e-20)
+            assert np.allclose(a.v[k], b.v[k], rtol=1e-12, atol=1e-30)
+            # one gradient for everyone: the moments are the same on every replica
+            assert np.all(a.m[k] == a.m[k][0]) and np.all(a.v[k] == a.v[k][0])
