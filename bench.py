@@ -42,12 +42,18 @@ FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
 
 
-def bytes_per_element(w: W.Workload) -> int:
-    """Algorithmic HBM bytes per replica-parameter-element of the fan-out kernel (fused converge adds none)."""
-    g = 2 if w.grad_dtype == W.DTYPE_BF16 else 4
+def bytes_per_element(w: W.Workload, shared_grad: bool = False, shared_state: bool = False) -> float:
+    """Algorithmic HBM bytes per replica-parameter-element of the fan-out kernel (fused converge adds none).
+
+    A shared gradient is read once per N replicas; shared moments are read and written once per N replicas.
+    The gradient replica-mean mode reads every replica's gradient, like the per-replica mode.
+    """
+    n = w.n_replicas
+    g = (2 if w.grad_dtype == W.DTYPE_BF16 else 4) / (n if shared_grad else 1)
     if w.optimizer == W.OPT_ADAMW:
-        return 12 + g + 12           # read theta, m, v, g; write theta, m, v
-    return 4 + g + 4                 # read theta, g; write theta
+        state = 16 / (n if shared_state else 1)      # m, v read and written
+        return 8 + g + state                         # theta read and written
+    return 8 + g
 
 
 def measured_peaks():
@@ -167,7 +173,7 @@ def pick_workload(name, torch, sync_interval=None):
     if sync_interval:
         from dataclasses import replace
         w = replace(w, sync_interval=sync_interval, name=f"{w.name}_T{sync_interval}")
-    need = w.n_replicas * w.arena_numel() * (bytes_per_element(w) - 12 if w.optimizer == W.OPT_ADAMW else 8)
+    need = w.n_replicas * w.arena_numel() * (14 if w.optimizer == W.OPT_ADAMW else 8)
     free, _ = torch.cuda.mem_get_info()
     note = None
     if need + (3 << 30) > free:
@@ -197,13 +203,18 @@ def run_ours(args):
     w, note = pick_workload(args.workload, torch, args.sync_interval)
     n, P = w.n_replicas, w.numel
     arena = StackedArena([t.numel for t in w.tensors], [t.group for t in w.tensors], n, w.optimizer, w.grad_dtype,
-                         device=f"cuda:{local}", align_elems=w.align_elems)
+                         device=f"cuda:{local}", align_elems=w.align_elems, shared_grad=args.shared_grad,
+                         shared_state=args.shared_state)
     D.fill(arena.param[0], R.param_key(w), 0, R.param_scale(w))
     for r in range(1, n):
         arena.param[r].copy_(arena.param[0])
-    for r in range(n):
-        D.fill(arena.grad[r], R.grad_key(w, 0, r), 0, R.grad_scale(w))
-    h = B.hdet_create(from_workload.config_for(w, fuse=1, device=local), arena.descriptors())
+    if args.shared_grad:
+        D.fill(arena.grad, R.grad_key(w, 0, 0), 0, R.grad_scale(w))
+    else:
+        for r in range(n):
+            D.fill(arena.grad[r], R.grad_key(w, 0, r), 0, R.grad_scale(w))
+    grad_mode = B.HDET_GRAD_REPLICA_MEAN if args.grad_mode == "mean" else B.HDET_GRAD_AS_GIVEN
+    h = B.hdet_create(from_workload.config_for(w, fuse=1, device=local, grad_mode=grad_mode), arena.descriptors())
     B.hdet_set_schedule(h, from_workload.schedule_for(w))
     stream = torch.cuda.current_stream()
     losses = [list(R.step_losses(w, i % w.total_steps)) for i in range(w.total_steps)]
@@ -243,12 +254,13 @@ def run_ours(args):
     # ---- end-to-end region: this step's gradients come from pinned host memory, the status word goes back --
     e2e_steps = max(1, min(args.steps, args.e2e_steps))
     host_grad = torch.empty(arena.p_pad, dtype=arena.grad.dtype).pin_memory()
-    host_grad.copy_(arena.grad[0].cpu())
-    h2d_bytes = n * arena.p_pad * arena.grad.element_size()
+    host_grad.copy_((arena.grad if args.shared_grad else arena.grad[0]).cpu())
+    n_grad_copies = 1 if args.shared_grad else n
+    h2d_bytes = n_grad_copies * arena.p_pad * arena.grad.element_size()
 
     def e2e_step():
-        for r in range(n):
-            arena.grad[r].copy_(host_grad, non_blocking=True)
+        for r in range(n_grad_copies):
+            (arena.grad if args.shared_grad else arena.grad[r]).copy_(host_grad, non_blocking=True)
         one_step()
         st = B.hdet_get_state(h, raise_on_nonfinite=False)   # reads the device status word back (synchronises)
         return st.device_status
@@ -282,12 +294,12 @@ def run_ours(args):
             torch.cuda.synchronize()
             return a.elapsed_time(b) / reps
 
-        bpe_step = bytes_per_element(w)
+        bpe_step = bytes_per_element(w, args.shared_grad, args.shared_state)
         for label, T, fuse, bpe_k in (("fanout_update", 1 << 40, 1, bpe_step),
                                       ("fanout_update_converge_fused", 1, 1, bpe_step),
                                       ("fanout_update_then_converge_unfused", 1, 0, bpe_step + 8)):
             wk = _replace(w, sync_interval=T, autolr=0)
-            hk = B.hdet_create(from_workload.config_for(wk, fuse=fuse, device=local), arena.descriptors())
+            hk = B.hdet_create(from_workload.config_for(wk, fuse=fuse, device=local, grad_mode=grad_mode), arena.descriptors())
             B.hdet_set_schedule(hk, from_workload.schedule_for(wk))
             ms = timed(lambda: B.hdet_step(hk, None, stream.cuda_stream))
             per_kernel[label] = {"ms": ms, "GB_per_s": bpe_k * n * P / ms / 1e6, "bytes_per_element": bpe_k}
@@ -301,12 +313,13 @@ def run_ours(args):
             dist.destroy_process_group()
         return
 
-    bpe = bytes_per_element(w)
+    bpe = bytes_per_element(w, args.shared_grad, args.shared_state)
     peak, peak_src = measured_peaks()
     launch_ms = statistics.mean(per_step_ms) / max(1, launches // args.steps)
     achieved = bpe * n * P / (launch_ms * 1e-3) / 1e9
     traffic, traffic_src = args.traffic_bytes, "command line" if args.traffic_bytes else None
-    if (traffic is None and NCU_DRAM_BYTES_PER_ELEMENT_ADAMW_BF16_CONVERGE and w.optimizer == W.OPT_ADAMW
+    plain_mode = not (args.shared_grad or args.shared_state or args.grad_mode == "mean")
+    if (traffic is None and plain_mode and NCU_DRAM_BYTES_PER_ELEMENT_ADAMW_BF16_CONVERGE and w.optimizer == W.OPT_ADAMW
             and w.grad_dtype == W.DTYPE_BF16 and w.sync_interval == 1):
         traffic = NCU_DRAM_BYTES_PER_ELEMENT_ADAMW_BF16_CONVERGE * n * P
         traffic_src = "ncu dram__bytes_read+write on the 25 M list, scaled by N*P (see profiles/)"
@@ -318,7 +331,8 @@ def run_ours(args):
         "config": {
             "workload": w.name, "n_replicas": n, "params_per_replica": P, "n_tensors": len(w.tensors),
             "optimizer": "adamw" if w.optimizer == W.OPT_ADAMW else "sgd", "sync_interval": w.sync_interval,
-            "alpha_lr": w.alpha_lr, "resident_gb": arena.resident_bytes() / 1e9,
+            "alpha_lr": w.alpha_lr, "grad_mode": args.grad_mode, "shared_grad": args.shared_grad,
+            "shared_moments": args.shared_state, "resident_gb": arena.resident_bytes() / 1e9,
             "l2_policy": "inputs larger than L2 (no flush)", "parallelism": f"{world} independent replicas of the job",
             "note": note,
         },
@@ -332,7 +346,7 @@ def run_ours(args):
                         "(+ hdet_autolr_update), device status word read back"},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "traffic": traffic, "traffic_source": traffic_src, "peak_source": peak_src,
-                     "kernel": "fanout_kernel (fused update+converge)" if w.sync_interval == 1 else "fanout_kernel",
+                     "kernel": ("fanout_shared_kernel" if args.shared_state else "fanout_kernel") + (" (fused update+converge)" if w.sync_interval == 1 else ""),
                      "bytes_per_element": bpe, "launch_ms": launch_ms},
         "per_kernel": per_kernel,
         "device_status": int(final_state.device_status),
@@ -375,6 +389,11 @@ def main():
     ap.add_argument("--workload", default="config4", choices=sorted(W.ALL_CONFIGS))
     ap.add_argument("--sync-interval", type=int, default=None,
                     help="override the workload's T (e.g. 1 to profile the fused update+converge kernel on a small list)")
+    ap.add_argument("--grad-mode", default="as_given", choices=["as_given", "mean"],
+                    help="mean: every replica steps with the on-device replica mean of the gradients")
+    ap.add_argument("--shared-grad", action="store_true", help="one gradient for all replicas (grad_stride 0)")
+    ap.add_argument("--shared-state", action="store_true",
+                    help="one pair of Adam moments for all replicas (needs --shared-grad or --grad-mode mean)")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-steps", type=int, default=30)
     ap.add_argument("--no-cpu-baseline", action="store_true")

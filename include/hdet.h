@@ -62,6 +62,7 @@ typedef enum {
 
 enum { HDET_OPT_SGD = 0, HDET_OPT_ADAMW = 1 };
 enum { HDET_DTYPE_F32 = 0, HDET_DTYPE_BF16 = 1 };
+enum { HDET_GRAD_AS_GIVEN = 0, HDET_GRAD_REPLICA_MEAN = 1 };
 enum { HDET_SCHED_CONSTANT = 0, HDET_SCHED_ONECYCLE_COS = 1, HDET_SCHED_ONECYCLE_LINEAR = 2 };
 
 typedef struct hdet_ctx* hdet_handle;
@@ -76,7 +77,10 @@ typedef struct {
   int64_t param_stride; /* elements between replicas of param (>= numel when N > 1)       */
   int64_t grad_stride;  /* elements between replicas of grad; 0 = one gradient shared by
                            every replica (the all-reduced gradient of Eq. 2)              */
-  int64_t state_stride; /* elements between replicas of both moments                     */
+  int64_t state_stride; /* elements between replicas of both moments; 0 = ONE pair of moments
+                           for all replicas, allowed only when every replica sees the same
+                           gradient (grad_stride 0, or grad_mode HDET_GRAD_REPLICA_MEAN), and
+                           then required of every tensor of the handle                    */
   int32_t group;        /* optimizer group, 0 .. n_groups-1                               */
   int32_t reserved;     /* set to 0                                                       */
 } hdet_tensor;
@@ -101,7 +105,11 @@ typedef struct {
                             the parameters); 0: update kernel then converge kernel        */
   uint64_t seed;         /* seed of the permutation generator                             */
   int32_t device;        /* CUDA device ordinal; ignored when n_tensors == 0              */
-  int32_t reserved;      /* set to 0                                                       */
+  int32_t grad_mode;     /* HDET_GRAD_AS_GIVEN: replica r steps with its own gradient (or the
+                            shared one when grad_stride is 0).  HDET_GRAD_REPLICA_MEAN: the
+                            kernel first averages the N per-replica gradients of a tile and
+                            every replica steps with that mean -- the single-GPU form of the
+                            gradient all-reduce in Algorithm 1's loop                      */
 } hdet_config;
 
 /* Base schedule and controller constants (Algorithm 1, Require).  Host arrays with
@@ -152,8 +160,9 @@ typedef struct {
  * tensors may be NULL only when n_tensors == 0.  On success *out receives the handle;
  * on failure *out is NULL and nothing is left allocated.
  * Errors: INVALID_ARG (NULL, N/G/T/alpha out of range, numel <= 0, group out of range,
- * stride < numel with N > 1, missing moments for AdamW), ALIGN, UNSUPPORTED (momentum
- * != 0), CUDA.
+ * stride < numel with N > 1, missing moments for AdamW, state_stride 0 without a common
+ * gradient), ALIGN, UNSUPPORTED (momentum != 0; some but not all tensors with
+ * state_stride 0), CUDA.
  */
 HDET_API int hdet_create(const hdet_config* cfg, const hdet_tensor* tensors, int64_t n_tensors, hdet_handle* out);
 

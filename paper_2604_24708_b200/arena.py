@@ -3,8 +3,8 @@
 Layout in HBM (one allocation per quantity, no per-tensor allocations):
 
     param      fp32  [N][P_pad]     replica r of tensor k at  r * P_pad + offset_k
-    exp_avg    fp32  [N][P_pad]     (AdamW only)
-    exp_avg_sq fp32  [N][P_pad]     (AdamW only)
+    exp_avg    fp32  [N][P_pad]     (AdamW only; [P_pad] when the moments are shared by all replicas)
+    exp_avg_sq fp32  [N][P_pad]     (AdamW only; likewise)
     grad       fp32 or bf16 [N][P_pad]   (or [P_pad] when one gradient is shared)
 
 Every offset_k is a multiple of ``align_elems`` (8 by default: 32 bytes of fp32, 16 bytes of
@@ -22,7 +22,8 @@ from . import binding as B
 
 class StackedArena:
     def __init__(self, numels: Sequence[int], groups: Sequence[int], n_replicas: int, optimizer: int,
-                 grad_dtype: int, device: str = "cuda:0", align_elems: int = 8, shared_grad: bool = False):
+                 grad_dtype: int, device: str = "cuda:0", align_elems: int = 8, shared_grad: bool = False,
+                 shared_state: bool = False):
         if not torch.cuda.is_available():
             raise RuntimeError("StackedArena needs a CUDA device (there is no CPU path)")
         self.numels = [int(x) for x in numels]
@@ -41,8 +42,10 @@ class StackedArena:
         gd = torch.bfloat16 if grad_dtype == B.HDET_DTYPE_BF16 else torch.float32
         self.param = torch.zeros((self.n, self.p_pad), dtype=torch.float32, device=self.device)
         adam = optimizer == B.HDET_OPT_ADAMW
-        self.exp_avg = torch.zeros_like(self.param) if adam else None
-        self.exp_avg_sq = torch.zeros_like(self.param) if adam else None
+        self.shared_state = bool(shared_state) and adam
+        sshape = (self.p_pad,) if self.shared_state else (self.n, self.p_pad)
+        self.exp_avg = torch.zeros(sshape, dtype=torch.float32, device=self.device) if adam else None
+        self.exp_avg_sq = torch.zeros(sshape, dtype=torch.float32, device=self.device) if adam else None
         self.shared_grad = bool(shared_grad)
         gshape = (self.p_pad,) if shared_grad else (self.n, self.p_pad)
         self.grad = torch.zeros(gshape, dtype=gd, device=self.device)
@@ -60,7 +63,7 @@ class StackedArena:
             t.numel = ne
             t.param_stride = self.p_pad
             t.grad_stride = 0 if self.shared_grad else self.p_pad
-            t.state_stride = self.p_pad
+            t.state_stride = 0 if self.shared_state else self.p_pad
             t.group = grp
             out.append(t)
         return out

@@ -22,6 +22,7 @@ HDET_ERR_NONFINITE = 6
 
 HDET_OPT_SGD, HDET_OPT_ADAMW = 0, 1
 HDET_DTYPE_F32, HDET_DTYPE_BF16 = 0, 1
+HDET_GRAD_AS_GIVEN, HDET_GRAD_REPLICA_MEAN = 0, 1
 HDET_SCHED_CONSTANT, HDET_SCHED_ONECYCLE_COS, HDET_SCHED_ONECYCLE_LINEAR = 0, 1, 2
 
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "lib", "libhdet.so")
@@ -48,7 +49,7 @@ class hdet_config(C.Structure):
         ("beta1", C.c_double), ("beta2", C.c_double), ("eps", C.c_double), ("momentum", C.c_double),
         ("alpha_lr", C.c_double), ("alpha_wd", C.c_double), ("sync_interval", C.c_int64),
         ("reshuffle", C.c_int32), ("fuse_converge", C.c_int32), ("seed", C.c_uint64),
-        ("device", C.c_int32), ("reserved", C.c_int32),
+        ("device", C.c_int32), ("grad_mode", C.c_int32),
     ]
 
 

@@ -46,6 +46,7 @@ struct hdet_ctx {
   int n_tiles = 0;
   int grid_fanout = 0;
   int grid_converge = 0;
+  bool shared_state = false;   // AdamW with one pair of moments for all replicas
   int64_t launches = 0;
   std::string error;
 };
@@ -140,11 +141,15 @@ int hdet_create(const hdet_config* cfg, const hdet_tensor* tensors, int64_t n_te
       return fail(nullptr, HDET_ERR_INVALID_ARG, "hdet_create: need 0 <= beta1, beta2 < 1 and eps >= 0");
   }
   if (cfg->momentum != 0.0) return fail(nullptr, HDET_ERR_UNSUPPORTED, "hdet_create: SGD momentum is not implemented");
+  if (cfg->grad_mode != HDET_GRAD_AS_GIVEN && cfg->grad_mode != HDET_GRAD_REPLICA_MEAN)
+    return fail(nullptr, HDET_ERR_INVALID_ARG, "hdet_create: unknown grad_mode");
 
   const int n = cfg->n_replicas;
   const size_t gsz = cfg->grad_dtype == HDET_DTYPE_BF16 ? 2 : 4;
   std::vector<TensorDesc> descs;
   std::vector<Tile> tiles;
+  int64_t n_shared_state = 0;
+  const bool adamw = cfg->optimizer == HDET_OPT_ADAMW;
   for (int64_t k = 0; k < n_tensors; ++k) {
     const hdet_tensor& t = tensors[k];
     char where[64];
@@ -156,8 +161,14 @@ int hdet_create(const hdet_config* cfg, const hdet_tensor* tensors, int64_t n_te
     if (t.group < 0 || t.group >= cfg->n_groups)
       return fail(nullptr, HDET_ERR_INVALID_ARG, std::string(where) + "group out of range");
     if (n > 1 && (t.param_stride < t.numel || (t.grad_stride != 0 && t.grad_stride < t.numel) ||
-                  (cfg->optimizer == HDET_OPT_ADAMW && t.state_stride < t.numel)))
+                  (adamw && t.state_stride != 0 && t.state_stride < t.numel)))
       return fail(nullptr, HDET_ERR_INVALID_ARG, std::string(where) + "a replica stride is smaller than numel");
+    if (n > 1 && adamw && t.state_stride == 0) {
+      if (t.grad_stride != 0 && cfg->grad_mode != HDET_GRAD_REPLICA_MEAN)
+        return fail(nullptr, HDET_ERR_INVALID_ARG, std::string(where) +
+                    "state_stride 0 (shared moments) needs a gradient common to all replicas");
+      ++n_shared_state;
+    }
     if (t.param_stride < 0 || t.grad_stride < 0 || t.state_stride < 0)
       return fail(nullptr, HDET_ERR_INVALID_ARG, std::string(where) + "negative stride");
     if (!aligned(t.param, 4) || !aligned(t.grad, gsz) || (t.exp_avg && !aligned(t.exp_avg, 4)) ||
@@ -184,11 +195,15 @@ int hdet_create(const hdet_config* cfg, const hdet_tensor* tensors, int64_t n_te
     for (int64_t j = 0; j < n_tiles_t; ++j) tiles.push_back(Tile{(int)k, (int)j});
   }
 
+  if (n_shared_state != 0 && n_shared_state != n_tensors)
+    return fail(nullptr, HDET_ERR_UNSUPPORTED, "hdet_create: state_stride 0 must be used by all tensors or by none");
+
   hdet_ctx* h = new (std::nothrow) hdet_ctx();
   if (!h) return fail(nullptr, HDET_ERR_INVALID_ARG, "hdet_create: out of host memory");
   h->cfg = *cfg;
   h->n_tensors = n_tensors;
   h->n_tiles = (int)tiles.size();
+  h->shared_state = n_shared_state != 0;
   spread_multipliers(n, cfg->alpha_lr, h->rho_lr);
   spread_multipliers(n, cfg->alpha_wd, h->rho_wd);
   for (int g = 0; g < HDET_MAX_GROUPS; ++g)
@@ -287,7 +302,8 @@ int hdet_step(hdet_handle h, const double* step_losses, void* stream, int32_t* d
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const bool fuse = ends_round && h->cfg.fuse_converge;
     LaunchPlan plan{h->d_tensors, h->d_tiles, h->n_tiles, h->grid_fanout, h->d_status};
-    cudaError_t e = launch_fanout(h->cfg.optimizer, h->cfg.grad_dtype, fuse, plan, s, st);
+    cudaError_t e = launch_fanout(h->cfg.optimizer, h->cfg.grad_dtype, fuse, h->cfg.grad_mode == HDET_GRAD_REPLICA_MEAN,
+                                  h->shared_state, plan, s, st);
     if (e != cudaSuccess) return fail_cuda(h, "hdet_step: fan-out launch", e);
     ++h->launches;
     if (ends_round && !fuse) {

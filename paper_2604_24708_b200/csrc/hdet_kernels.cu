@@ -59,16 +59,22 @@ __device__ __forceinline__ float load_scalar(const __nv_bfloat16* p) {
 }
 
 // ---- scalar path: elements [begin, end) of one tensor, any alignment -----------------------
-template <typename GradT, bool kAdam, bool kConv>
+template <typename GradT, bool kAdam, bool kConv, bool kMean>
 __device__ void range_scalar(const TensorDesc& td, long long begin, long long end, const StepScalars& s,
                              const AdamConsts& c, bool& bad) {
   const int n = s.n_replicas;
   const GradT* grad = static_cast<const GradT*>(td.grad);
   for (long long e = begin + threadIdx.x; e < end; e += kThreads) {
     double sum = 0.0;
+    float gbar = 0.f;
+    if (kMean) {
+      double acc = 0.0;
+      for (int r = 0; r < n; ++r) acc += (double)load_scalar(grad + r * td.grad_stride + e);
+      gbar = (float)(acc * s.inv_n);
+    }
     for (int r = 0; r < n; ++r) {
       float th = __ldcs(td.param + r * td.param_stride + e);
-      const float g = load_scalar(grad + r * td.grad_stride + e);
+      const float g = kMean ? gbar : load_scalar(grad + r * td.grad_stride + e);
       if (kAdam) {
         float m = __ldcs(td.exp_avg + r * td.state_stride + e);
         float v = __ldcs(td.exp_avg_sq + r * td.state_stride + e);
@@ -90,6 +96,35 @@ __device__ void range_scalar(const TensorDesc& td, long long begin, long long en
 }
 
 // ---- vector path ---------------------------------------------------------------------------
+// gbar[k][q] = (1/N) sum_r g_r for the thread's vectors of one tile.  The sum is taken in fp64 (exact for
+// bf16 gradients, correctly rounded for fp32 ones): where the g_r cancel, Adam's m / (sqrt(v) + eps) is
+// sensitive to the low bits of the mean.
+template <typename GradT>
+__device__ __forceinline__ void mean_gradient(const GradT* Gp, long long gs, const int (&idx)[kTileVecs],
+                                              const bool (&ok)[kTileVecs], int n, double inv_n,
+                                              float (&gbar)[kTileVecs][4]) {
+  double acc[kTileVecs][4];
+#pragma unroll
+  for (int k = 0; k < kTileVecs; ++k)
+#pragma unroll
+    for (int q = 0; q < 4; ++q) acc[k][q] = 0.0;
+#pragma unroll 4
+  for (int r = 0; r < n; ++r) {
+#pragma unroll
+    for (int k = 0; k < kTileVecs; ++k) {
+      if (!ok[k]) continue;
+      float g[4];
+      unpack(load_raw(Gp + r * gs + idx[k]), g);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) acc[k][q] += (double)g[q];
+    }
+  }
+#pragma unroll
+  for (int k = 0; k < kTileVecs; ++k)
+#pragma unroll
+    for (int q = 0; q < 4; ++q) gbar[k][q] = (float)(acc[k][q] * inv_n);
+}
+
 template <typename GradT, bool kAdam>
 struct ReplicaRegs {
   float4 th[kTileVecs];
@@ -99,7 +134,7 @@ struct ReplicaRegs {
 };
 
 // Processes `nvec` float4 vectors starting at element `off` of the tensor.  kFull: nvec == kThreads*kTileVecs.
-template <typename GradT, bool kAdam, bool kConv, bool kFull>
+template <typename GradT, bool kAdam, bool kConv, bool kMean, bool kFull>
 __device__ __forceinline__ void tile_vector(const TensorDesc& td, long long off, int nvec, const StepScalars& s,
                                             const AdamConsts& c, bool& bad) {
   using Regs = ReplicaRegs<GradT, kAdam>;
@@ -129,7 +164,7 @@ __device__ __forceinline__ void tile_vector(const TensorDesc& td, long long off,
           b.m[k] = __ldcs(reinterpret_cast<const float4*>(M + r * ss + idx[k]));
           b.v[k] = __ldcs(reinterpret_cast<const float4*>(V + r * ss + idx[k]));
         }
-        b.g[k] = load_raw(Gp + r * gs + idx[k]);
+        if (!kMean) b.g[k] = load_raw(Gp + r * gs + idx[k]);
       } else {
         b.th[k] = make_float4(0.f, 0.f, 0.f, 0.f);
         if (kAdam) { b.m[k] = b.th[k]; b.v[k] = b.th[k]; }
@@ -137,6 +172,13 @@ __device__ __forceinline__ void tile_vector(const TensorDesc& td, long long off,
       }
     }
   };
+
+  // Replica 0 is requested first; then the gradient replica-mean (the all-reduced gradient of
+  // Algorithm 1) is formed once per tile while those loads are in flight.
+  Regs a, b;
+  load(a, 0);
+  float gbar[kTileVecs][4];
+  if constexpr (kMean) mean_gradient<GradT>(Gp, gs, idx, ok, n, s.inv_n, gbar);
 
   double sum[kConv ? kTileVecs : 1][4];
   if (kConv) {
@@ -152,7 +194,12 @@ __device__ __forceinline__ void tile_vector(const TensorDesc& td, long long off,
 #pragma unroll
     for (int k = 0; k < kTileVecs; ++k) {
       float g[4];
-      unpack(b.g[k], g);
+      if constexpr (kMean) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) g[q] = gbar[k][q];
+      } else {
+        unpack(b.g[k], g);
+      }
       float th[4] = {b.th[k].x, b.th[k].y, b.th[k].z, b.th[k].w};
       if (kAdam) {
         float m[4] = {b.m[k].x, b.m[k].y, b.m[k].z, b.m[k].w};
@@ -179,8 +226,6 @@ __device__ __forceinline__ void tile_vector(const TensorDesc& td, long long off,
   };
 
   // Two-stage register pipeline over the replica axis.
-  Regs a, b;
-  load(a, 0);
   int r = 0;
   for (; r + 1 < n; r += 2) {
     load(b, r + 1);
@@ -202,7 +247,7 @@ __device__ __forceinline__ void tile_vector(const TensorDesc& td, long long off,
   }
 }
 
-template <typename GradT, bool kAdam, bool kConv>
+template <typename GradT, bool kAdam, bool kConv, bool kMean>
 __global__ void __launch_bounds__(kThreads, 2)
 fanout_kernel(const __grid_constant__ LaunchPlan plan, const __grid_constant__ StepScalars s) {
   const AdamConsts c{s.one_minus_beta1, s.one_minus_beta2, s.rsqrt_bc2, s.eps};
@@ -215,18 +260,199 @@ fanout_kernel(const __grid_constant__ LaunchPlan plan, const __grid_constant__ S
     const int len = rest < kTileElems ? (int)rest : kTileElems;
     if (td.vec) {
       if (len == kTileElems) {
-        tile_vector<GradT, kAdam, kConv, true>(td, off, kThreads * kTileVecs, s, c, bad);
+        tile_vector<GradT, kAdam, kConv, kMean, true>(td, off, kThreads * kTileVecs, s, c, bad);
       } else {
         const int nvec = len >> 2;
-        if (nvec) tile_vector<GradT, kAdam, kConv, false>(td, off, nvec, s, c, bad);
-        if (len & 3) range_scalar<GradT, kAdam, kConv>(td, off + 4ll * nvec, off + len, s, c, bad);
+        if (nvec) tile_vector<GradT, kAdam, kConv, kMean, false>(td, off, nvec, s, c, bad);
+        if (len & 3) range_scalar<GradT, kAdam, kConv, kMean>(td, off + 4ll * nvec, off + len, s, c, bad);
       }
     } else {
-      range_scalar<GradT, kAdam, kConv>(td, off, off + len, s, c, bad);
+      range_scalar<GradT, kAdam, kConv, kMean>(td, off, off + len, s, c, bad);
     }
   }
   if (bad) atomicOr(plan.status, 1u);
 }
+
+// ---- AdamW with ONE pair of moments for all replicas ------------------------------------------------
+// When every replica sees the same gradient (a shared gradient as in Eq. 2, or the replica mean of
+// Algorithm 1's gradient all-reduce) the Adam moments are identical on all replicas: they are stored
+// once (state_stride = 0), updated once per tile, and the step direction u = m / (sqrt(v)/sqrt(bc2) + eps)
+// is computed once; each replica then costs two fused multiply-adds per element:
+//   theta_r <- theta_r - (lr_r wd_r) theta_r - (lr_r / bc1) u.
+// Bytes per replica-element: 8 (theta) + (gradient + 16) / N, or 8 + gradient + 16 / N with the mean.
+constexpr int kBatch = 4;  // replicas of one vector loaded together; two batches are in flight
+
+template <typename GradT, bool kConv, bool kMean>
+__device__ void range_scalar_shared(const TensorDesc& td, long long begin, long long end, const StepScalars& s,
+                                    const AdamConsts& c, bool& bad) {
+  const int n = s.n_replicas;
+  const GradT* grad = static_cast<const GradT*>(td.grad);
+  for (long long e = begin + threadIdx.x; e < end; e += kThreads) {
+    float g;
+    if (kMean) {
+      double acc = 0.0;
+      for (int r = 0; r < n; ++r) acc += (double)load_scalar(grad + r * td.grad_stride + e);
+      g = (float)(acc * s.inv_n);
+    } else {
+      g = load_scalar(grad + e);
+    }
+    float m = __ldcs(td.exp_avg + e), v = __ldcs(td.exp_avg_sq + e);
+    m = fmaf(c.one_minus_beta1, g - m, m);
+    v = fmaf(c.one_minus_beta2, fmaf(g, g, -v), v);
+    const float u = m / fmaf(sqrtf(v), c.rsqrt_bc2, c.eps);
+    __stcs(td.exp_avg + e, m);
+    __stcs(td.exp_avg_sq + e, v);
+    double sum = 0.0;
+    for (int r = 0; r < n; ++r) {
+      float th = __ldcs(td.param + r * td.param_stride + e);
+      th = fmaf(-s.step[td.group][r], u, fmaf(-s.lr_wd[td.group][r], th, th));
+      bad |= not_finite(th);
+      if (kConv) sum += (double)th;
+      else __stcs(td.param + r * td.param_stride + e, th);
+    }
+    if (kConv) {
+      const float mean = (float)(sum * s.inv_n);
+      for (int r = 0; r < n; ++r) __stcs(td.param + r * td.param_stride + e, mean);
+    }
+  }
+}
+
+template <typename GradT, bool kConv, bool kMean, bool kFull>
+__device__ __forceinline__ void tile_vector_shared(const TensorDesc& td, long long off, int nvec,
+                                                   const StepScalars& s, const AdamConsts& c, bool& bad) {
+  const int n = s.n_replicas;
+  const int grp = td.group;
+  float* const P = td.param + off;
+  float* const M = td.exp_avg + off;
+  float* const V = td.exp_avg_sq + off;
+  const GradT* const Gp = static_cast<const GradT*>(td.grad) + off;
+  const long long ps = td.param_stride;
+
+  int idx[kTileVecs];
+  bool ok[kTileVecs];
+#pragma unroll
+  for (int k = 0; k < kTileVecs; ++k) {
+    const int j = k * kThreads + threadIdx.x;
+    idx[k] = j * 4;
+    ok[k] = kFull || j < nvec;
+  }
+
+  using Batch = float4[kBatch];
+  auto load_batch = [&](Batch& buf, int r0, int at, bool valid) {
+#pragma unroll
+    for (int j = 0; j < kBatch; ++j)
+      buf[j] = (valid && r0 + j < n) ? __ldcs(reinterpret_cast<const float4*>(P + (r0 + j) * ps + at))
+                                     : make_float4(0.f, 0.f, 0.f, 0.f);
+  };
+
+  // The first parameters are requested before the gradient and the moments are consumed.
+  Batch a, b;
+  load_batch(a, 0, idx[0], ok[0]);
+
+  // Step direction u = m' / (sqrt(v')/sqrt(bc2) + eps), once per element for all replicas.
+  float u[kTileVecs][4];
+  if constexpr (kMean) {
+    mean_gradient<GradT>(Gp, td.grad_stride, idx, ok, n, s.inv_n, u);
+  } else {
+#pragma unroll
+    for (int k = 0; k < kTileVecs; ++k) {
+      if (ok[k]) {
+        unpack(load_raw(Gp + idx[k]), u[k]);
+      } else {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) u[k][q] = 0.f;
+      }
+    }
+  }
+#pragma unroll
+  for (int k = 0; k < kTileVecs; ++k) {
+    float4 m4 = make_float4(0.f, 0.f, 0.f, 0.f), v4 = m4;
+    if (ok[k]) {
+      m4 = __ldcs(reinterpret_cast<const float4*>(M + idx[k]));
+      v4 = __ldcs(reinterpret_cast<const float4*>(V + idx[k]));
+    }
+    float m[4] = {m4.x, m4.y, m4.z, m4.w};
+    float v[4] = {v4.x, v4.y, v4.z, v4.w};
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const float g = u[k][q];
+      m[q] = fmaf(c.one_minus_beta1, g - m[q], m[q]);
+      v[q] = fmaf(c.one_minus_beta2, fmaf(g, g, -v[q]), v[q]);
+      u[k][q] = m[q] / fmaf(sqrtf(v[q]), c.rsqrt_bc2, c.eps);
+    }
+    if (ok[k]) {
+      __stcs(reinterpret_cast<float4*>(M + idx[k]), make_float4(m[0], m[1], m[2], m[3]));
+      __stcs(reinterpret_cast<float4*>(V + idx[k]), make_float4(v[0], v[1], v[2], v[3]));
+    }
+  }
+
+  // Replicas: per vector, batches of kBatch replicas, the next batch in flight while one is updated.
+#pragma unroll
+  for (int k = 0; k < kTileVecs; ++k) {
+    double sum[4] = {0.0, 0.0, 0.0, 0.0};
+    auto update_batch = [&](Batch& buf, int r0) {
+#pragma unroll
+      for (int j = 0; j < kBatch; ++j) {
+        const int r = r0 + j;
+        if (r < n) {
+          const float lr_wd = s.lr_wd[grp][r];
+          const float step = s.step[grp][r];
+          float th[4] = {buf[j].x, buf[j].y, buf[j].z, buf[j].w};
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            th[q] = fmaf(-step, u[k][q], fmaf(-lr_wd, th[q], th[q]));
+            bad |= not_finite(th[q]);
+          }
+          if (kConv) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q) sum[q] += (double)th[q];
+          } else if (ok[k]) {
+            __stcs(reinterpret_cast<float4*>(P + r * ps + idx[k]), make_float4(th[0], th[1], th[2], th[3]));
+          }
+        }
+      }
+    };
+    if (k > 0) load_batch(a, 0, idx[k], ok[k]);
+    for (int r0 = 0; r0 < n; r0 += 2 * kBatch) {
+      if (r0 + kBatch < n) load_batch(b, r0 + kBatch, idx[k], ok[k]);
+      update_batch(a, r0);
+      if (r0 + 2 * kBatch < n) load_batch(a, r0 + 2 * kBatch, idx[k], ok[k]);
+      if (r0 + kBatch < n) update_batch(b, r0 + kBatch);
+    }
+    if (kConv && ok[k]) {
+      const float4 mean = make_float4((float)(sum[0] * s.inv_n), (float)(sum[1] * s.inv_n),
+                                      (float)(sum[2] * s.inv_n), (float)(sum[3] * s.inv_n));
+      for (int rr = 0; rr < n; ++rr) __stcs(reinterpret_cast<float4*>(P + rr * ps + idx[k]), mean);
+    }
+  }
+}
+
+template <typename GradT, bool kConv, bool kMean>
+__global__ void __launch_bounds__(kThreads, 2)
+fanout_shared_kernel(const __grid_constant__ LaunchPlan plan, const __grid_constant__ StepScalars s) {
+  const AdamConsts c{s.one_minus_beta1, s.one_minus_beta2, s.rsqrt_bc2, s.eps};
+  bool bad = false;
+  for (int t = blockIdx.x; t < plan.n_tiles; t += gridDim.x) {
+    const Tile tile = plan.tiles[t];
+    const TensorDesc td = plan.tensors[tile.tensor];
+    const long long off = (long long)tile.tile * kTileElems;
+    const long long rest = td.numel - off;
+    const int len = rest < kTileElems ? (int)rest : kTileElems;
+    if (td.vec) {
+      if (len == kTileElems) {
+        tile_vector_shared<GradT, kConv, kMean, true>(td, off, kThreads * kTileVecs, s, c, bad);
+      } else {
+        const int nvec = len >> 2;
+        if (nvec) tile_vector_shared<GradT, kConv, kMean, false>(td, off, nvec, s, c, bad);
+        if (len & 3) range_scalar_shared<GradT, kConv, kMean>(td, off + 4ll * nvec, off + len, s, c, bad);
+      }
+    } else {
+      range_scalar_shared<GradT, kConv, kMean>(td, off, off + len, s, c, bad);
+    }
+  }
+  if (bad) atomicOr(plan.status, 1u);
+}
+
 
 // ---- stand-alone converge (Eq. 3) -------------------------------------------------------------
 __global__ void __launch_bounds__(kThreads, 4)
@@ -258,27 +484,42 @@ converge_kernel(const __grid_constant__ LaunchPlan plan, int n, double inv_n) {
   }
 }
 
-template <typename GradT, bool kAdam, bool kConv>
+template <typename GradT, bool kAdam, bool kConv, bool kMean>
 cudaError_t launch_one(const LaunchPlan& plan, const StepScalars& s, cudaStream_t stream) {
-  fanout_kernel<GradT, kAdam, kConv><<<plan.grid, kThreads, 0, stream>>>(plan, s);
+  fanout_kernel<GradT, kAdam, kConv, kMean><<<plan.grid, kThreads, 0, stream>>>(plan, s);
   return cudaGetLastError();
+}
+
+template <typename GradT, bool kConv, bool kMean>
+cudaError_t launch_shared(const LaunchPlan& plan, const StepScalars& s, cudaStream_t stream) {
+  fanout_shared_kernel<GradT, kConv, kMean><<<plan.grid, kThreads, 0, stream>>>(plan, s);
+  return cudaGetLastError();
+}
+
+template <typename GradT, bool kConv, bool kMean>
+cudaError_t pick_state(bool adam, bool shared_state, const LaunchPlan& plan, const StepScalars& s, cudaStream_t st) {
+  if (adam && shared_state) return launch_shared<GradT, kConv, kMean>(plan, s, st);
+  return adam ? launch_one<GradT, true, kConv, kMean>(plan, s, st) : launch_one<GradT, false, kConv, kMean>(plan, s, st);
+}
+
+template <typename GradT>
+cudaError_t pick_flags(bool adam, bool converge, bool mean, bool shared_state, const LaunchPlan& plan,
+                       const StepScalars& s, cudaStream_t st) {
+  if (converge) return mean ? pick_state<GradT, true, true>(adam, shared_state, plan, s, st)
+                            : pick_state<GradT, true, false>(adam, shared_state, plan, s, st);
+  return mean ? pick_state<GradT, false, true>(adam, shared_state, plan, s, st)
+              : pick_state<GradT, false, false>(adam, shared_state, plan, s, st);
 }
 
 }  // namespace
 
-cudaError_t launch_fanout(int optimizer, int grad_dtype, bool converge, const LaunchPlan& plan,
-                          const StepScalars& s, cudaStream_t stream) {
+cudaError_t launch_fanout(int optimizer, int grad_dtype, bool converge, bool grad_mean, bool shared_state,
+                          const LaunchPlan& plan, const StepScalars& s, cudaStream_t stream) {
   if (plan.n_tiles == 0) return cudaSuccess;
   const bool adam = optimizer == HDET_OPT_ADAMW;
-  const bool bf16 = grad_dtype == HDET_DTYPE_BF16;
-  if (adam) {
-    if (bf16) return converge ? launch_one<__nv_bfloat16, true, true>(plan, s, stream)
-                              : launch_one<__nv_bfloat16, true, false>(plan, s, stream);
-    return converge ? launch_one<float, true, true>(plan, s, stream) : launch_one<float, true, false>(plan, s, stream);
-  }
-  if (bf16) return converge ? launch_one<__nv_bfloat16, false, true>(plan, s, stream)
-                            : launch_one<__nv_bfloat16, false, false>(plan, s, stream);
-  return converge ? launch_one<float, false, true>(plan, s, stream) : launch_one<float, false, false>(plan, s, stream);
+  if (grad_dtype == HDET_DTYPE_BF16)
+    return pick_flags<__nv_bfloat16>(adam, converge, grad_mean, shared_state, plan, s, stream);
+  return pick_flags<float>(adam, converge, grad_mean, shared_state, plan, s, stream);
 }
 
 cudaError_t launch_converge(const LaunchPlan& plan, int n_replicas, cudaStream_t stream) {

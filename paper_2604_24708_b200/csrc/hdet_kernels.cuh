@@ -22,7 +22,7 @@ struct TensorDesc {
   long long numel;
   long long param_stride;
   long long grad_stride;
-  long long state_stride;
+  long long state_stride;  // 0: one pair of moments shared by all replicas
   int group;
   int vec;  // 1: pointers and strides allow 128-bit accesses
 };
@@ -54,8 +54,10 @@ struct LaunchPlan {
 
 // Fan-out update of every replica of every tile (Eq. 2 or Adam); with `converge` the
 // replica mean (Eq. 3) is formed from the updated values and written to all replicas.
-cudaError_t launch_fanout(int optimizer, int grad_dtype, bool converge, const LaunchPlan& plan,
-                          const StepScalars& s, cudaStream_t stream);
+// `grad_mean`: every replica steps with the replica mean of the gradients (Algorithm 1's gradient
+// all-reduce).  `shared_state`: AdamW with one pair of moments for all replicas (state_stride 0).
+cudaError_t launch_fanout(int optimizer, int grad_dtype, bool converge, bool grad_mean, bool shared_state,
+                          const LaunchPlan& plan, const StepScalars& s, cudaStream_t stream);
 
 // Stand-alone Eq. 3.
 cudaError_t launch_converge(const LaunchPlan& plan, int n_replicas, cudaStream_t stream);

@@ -11,9 +11,9 @@ from oracle import hdet_oracle as O
 
 
 # ----------------------------------------------------------------------------- library side
-def lib_config(B, w: W.Workload, fuse: int = 1, device: int = 0):
+def lib_config(B, w: W.Workload, fuse: int = 1, device: int = 0, grad_mode: int = 0):
     from paper_2604_24708_b200 import from_workload
-    return from_workload.config_for(w, fuse, device)
+    return from_workload.config_for(w, fuse, device, grad_mode)
 
 
 def lib_schedule(B, w: W.Workload):
@@ -24,7 +24,8 @@ def lib_schedule(B, w: W.Workload):
 class GpuRun:
     """The workload resident on the GPU, stepped through the C ABI."""
 
-    def __init__(self, w: W.Workload, fuse: int = 1, shared_grad: bool = False, device: int = 0):
+    def __init__(self, w: W.Workload, fuse: int = 1, shared_grad: bool = False, device: int = 0,
+                 grad_mean: bool = False, shared_state: bool = False):
         import torch
         from hdet_inputs import device as D
         from paper_2604_24708_b200 import binding as B
@@ -33,12 +34,12 @@ class GpuRun:
         self.B, self.D, self.torch, self.w = B, D, torch, w
         self.arena = StackedArena([t.numel for t in w.tensors], [t.group for t in w.tensors], w.n_replicas,
                                   w.optimizer, w.grad_dtype, device=f"cuda:{device}", align_elems=w.align_elems,
-                                  shared_grad=shared_grad)
+                                  shared_grad=shared_grad, shared_state=shared_state)
         assert self.arena.offsets == w.arena_offsets()
         D.fill(self.arena.param[0], R.param_key(w), 0, R.param_scale(w))
         for r in range(1, w.n_replicas):
             self.arena.param[r].copy_(self.arena.param[0])
-        self.h = B.hdet_create(lib_config(B, w, fuse, device), self.arena.descriptors())
+        self.h = B.hdet_create(lib_config(B, w, fuse, device, 1 if grad_mean else 0), self.arena.descriptors())
         B.hdet_set_schedule(self.h, lib_schedule(B, w))
         self.i = 0
 
@@ -71,6 +72,8 @@ class GpuRun:
         """[N, n] values of tensor k, elements start .. start+n-1, copied to the host."""
         t = {"param": self.arena.param, "m": self.arena.exp_avg, "v": self.arena.exp_avg_sq}[which]
         off = self.arena.offsets[k] + start
+        if t.dim() == 1:                       # moments shared by all replicas
+            return t[None, off:off + n].float().cpu().numpy()
         return t[:, off:off + n].float().cpu().numpy()
 
     def close(self) -> None:
@@ -85,26 +88,28 @@ class GpuRun:
 Slab = Tuple[int, int, int]   # (tensor index, first element inside the tensor, length)
 
 
-def oracle_for(w: W.Workload, params: Sequence[np.ndarray], groups: Sequence[int]) -> O.HdetOracle:
+def oracle_for(w: W.Workload, params: Sequence[np.ndarray], groups: Sequence[int],
+               grad_mean: bool = False) -> O.HdetOracle:
     return O.HdetOracle(
         params, groups, w.n_groups, optimizer=w.optimizer, total_steps=w.total_steps, sched_kind=w.sched_kind,
         max_lr=list(w.max_lr), weight_decay=list(w.weight_decay), pct_start=w.pct_start, div_factor=w.div_factor,
         final_div_factor=w.final_div_factor, alpha_lr=w.alpha_lr, alpha_wd=w.alpha_wd,
         sync_interval=w.sync_interval, autolr=bool(w.autolr), warmup_steps=w.warmup_steps, ctrl_beta=w.ctrl_beta,
         ctrl_sigma=w.ctrl_sigma, ctrl_lambda=w.ctrl_lambda, f_div=w.f_div, f_final=w.f_final,
-        reshuffle=bool(w.reshuffle), seed=w.seed, beta1=w.beta1, beta2=w.beta2, eps=w.eps, n_replicas=w.n_replicas)
+        reshuffle=bool(w.reshuffle), seed=w.seed, beta1=w.beta1, beta2=w.beta2, eps=w.eps, n_replicas=w.n_replicas,
+        grad_mean=grad_mean)
 
 
 class OracleRun:
     """The oracle over chosen element ranges (slabs) of the workload, with the same seeded inputs."""
 
-    def __init__(self, w: W.Workload, slabs: Sequence[Slab], shared_grad: bool = False):
+    def __init__(self, w: W.Workload, slabs: Sequence[Slab], shared_grad: bool = False, grad_mean: bool = False):
         self.w, self.slabs, self.shared_grad = w, list(slabs), shared_grad
         offs = w.arena_offsets()
         self.starts = [offs[k] + s for (k, s, n) in self.slabs]
         params = [np.tile(R.param_slab(w, a, n).astype(np.float64), (w.n_replicas, 1))
                   for a, (k, s, n) in zip(self.starts, self.slabs)]
-        self.o = oracle_for(w, params, [w.tensors[k].group for (k, s, n) in self.slabs])
+        self.o = oracle_for(w, params, [w.tensors[k].group for (k, s, n) in self.slabs], grad_mean=grad_mean)
         self.i = 0
 
     def grads(self, step: int) -> List[np.ndarray]:
@@ -164,7 +169,11 @@ def compare_slabs(g: GpuRun, o: OracleRun, tol: float, check_moments: bool = Tru
         if adam and check_moments:
             pairs += [("m", o.o.m[idx]), ("v", o.o.v[idx])]
         for name, ref in pairs:
-            e = rel_err(g.slab(name, k, s, n), ref).max()
+            got = g.slab(name, k, s, n)
+            if got.shape[0] == 1 and ref.shape[0] > 1:       # shared moments: every oracle replica must agree
+                assert np.all(ref == ref[0:1]), f"oracle {name} differs between replicas although the gradient is common"
+                ref = ref[0:1]
+            e = rel_err(got, ref).max()
             assert e <= tol, f"{name} of tensor {k} [{s}:{s + n}] at step {g.i}: rel err {e:.3e} > {tol:.1e}"
             worst = max(worst, float(e))
     return worst

@@ -19,10 +19,10 @@ TOL_ONE_STEP = 1e-6
 TOL_FULL_RUN = 1e-5
 
 
-def _lockstep(w, slabs, steps=None, fuse=1, shared_grad=False, check_every=None):
+def _lockstep(w, slabs, steps=None, fuse=1, shared_grad=False, check_every=None, grad_mean=False, shared_state=False):
     """Runs both sides for `steps` updates; checks after the first update, at chosen steps and at the end."""
-    g = H.GpuRun(w, fuse=fuse, shared_grad=shared_grad)
-    o = H.OracleRun(w, slabs, shared_grad=shared_grad)
+    g = H.GpuRun(w, fuse=fuse, shared_grad=shared_grad, grad_mean=grad_mean, shared_state=shared_state)
+    o = H.OracleRun(w, slabs, shared_grad=shared_grad, grad_mean=grad_mean)
     steps = steps or w.total_steps
     worst = 0.0
     try:
@@ -89,8 +89,8 @@ def test_shared_gradient_stride_zero():
     _lockstep(w, H.whole_tensor_slabs(w), shared_grad=True, check_every=4)
 
 
-def _final_arena(w, fuse=1, shared_grad=False, steps=None):
-    g = H.GpuRun(w, fuse=fuse, shared_grad=shared_grad)
+def _final_arena(w, fuse=1, shared_grad=False, steps=None, grad_mean=False, shared_state=False):
+    g = H.GpuRun(w, fuse=fuse, shared_grad=shared_grad, grad_mean=grad_mean, shared_state=shared_state)
     for i in range(steps or w.total_steps):
         g.step(g.perm0())
     a = g.arena
@@ -110,6 +110,46 @@ def test_fused_converge_equals_update_then_converge_bitwise_and_runs_are_determi
         assert torch.equal(a, b)
         assert torch.equal(a, c)
     assert l1 == w.total_steps and l2 == w.total_steps + w.total_steps // w.sync_interval
+
+
+@pytest.mark.parametrize("optimizer,grad_dtype", [(W.OPT_ADAMW, W.DTYPE_BF16), (W.OPT_ADAMW, W.DTYPE_F32),
+                                                   (W.OPT_SGD, W.DTYPE_F32), (W.OPT_SGD, W.DTYPE_BF16)])
+@pytest.mark.parametrize("align", [8, 1])
+def test_gradient_replica_mean_every_element(optimizer, grad_dtype, align):
+    """grad_mode = replica mean (Algorithm 1's gradient all-reduce on the device), per-replica moments."""
+    w = W.ragged_workload(n_replicas=5, optimizer=optimizer, grad_dtype=grad_dtype, align_elems=align)
+    _lockstep(w, H.whole_tensor_slabs(w), check_every=1, grad_mean=True)
+
+
+@pytest.mark.parametrize("grad_dtype", [W.DTYPE_BF16, W.DTYPE_F32])
+@pytest.mark.parametrize("align", [8, 1])
+@pytest.mark.parametrize("mode", ["shared_grad", "mean"])
+@pytest.mark.parametrize("n", [1, 2, 3, 4, 5, 8, 9, 32])
+def test_shared_moments_every_element(grad_dtype, align, mode, n):
+    """One pair of Adam moments for all replicas (state_stride 0), with a shared gradient or the replica mean."""
+    w = W.ragged_workload(n_replicas=n, grad_dtype=grad_dtype, align_elems=align, numels=(4099, 7, 2048, 1, 6150))
+    _lockstep(w, H.whole_tensor_slabs(w), check_every=3, shared_grad=(mode == "shared_grad"),
+              grad_mean=(mode == "mean"), shared_state=True)
+
+
+def test_shared_moments_kernel_equals_per_replica_moments_bitwise():
+    import torch
+    w = W.ragged_workload(n_replicas=6, numels=(4097, 2048, 33, 12289))
+    per_replica, _ = _final_arena(w, shared_grad=True)
+    shared, _ = _final_arena(w, shared_grad=True, shared_state=True)
+    assert torch.equal(per_replica[0], shared[0])
+    for a, b in zip(per_replica[1:], shared[1:]):
+        assert torch.equal(a, b[None].expand_as(a))
+    fused, _ = _final_arena(w, shared_grad=True, shared_state=True, fuse=0)
+    assert torch.equal(fused[0], shared[0])
+
+
+def test_config2_shape_with_gradient_mean_and_shared_moments_sampled():
+    """The paper's own arrangement on one GPU: one all-reduced gradient, N rates, moments stored once; 300 updates."""
+    w = replace(W.config2(), total_steps=300, warmup_steps=90)
+    slabs = [(k, 0, min(2048, t.numel)) for k, t in enumerate(w.tensors) if k % 4 < 2]
+    slabs += [(0, 2097152 - 4096, 4096), (10, 1024 * 1024 + 2048 * 7, 2048)]
+    _lockstep(w, slabs, check_every=100, grad_mean=True, shared_state=True)
 
 
 def test_alpha_zero_keeps_replicas_bitwise_identical():

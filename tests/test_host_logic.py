@@ -96,6 +96,16 @@ def test_create_rejects_momentum_and_bad_tensors_without_touching_a_device():
         with pytest.raises(B.HdetError) as e:
             B.hdet_create(_cfg(), [tens(**kw)])
         assert e.value.status == status, kw
+    # shared moments (state_stride 0) need a gradient common to all replicas, and all tensors must agree
+    with pytest.raises(B.HdetError) as e:
+        B.hdet_create(_cfg(), [tens(state_stride=0)])
+    assert e.value.status == B.HDET_ERR_INVALID_ARG and "shared moments" in e.value.message
+    with pytest.raises(B.HdetError) as e:
+        B.hdet_create(_cfg(), [tens(state_stride=0, grad_stride=0), tens(grad_stride=0)])
+    assert e.value.status == B.HDET_ERR_UNSUPPORTED
+    with pytest.raises(B.HdetError) as e:
+        B.hdet_create(_cfg(grad_mode=7), [])
+    assert e.value.status == B.HDET_ERR_INVALID_ARG
     # NULL cfg / NULL out through the raw ABI
     lib = B.raw_library()
     h = C.c_void_p()
