@@ -280,7 +280,8 @@ fanout_kernel(const __grid_constant__ LaunchPlan plan, const __grid_constant__ S
 // is computed once; each replica then costs two fused multiply-adds per element:
 //   theta_r <- theta_r - (lr_r wd_r) theta_r - (lr_r / bc1) u.
 // Bytes per replica-element: 8 (theta) + (gradient + 16) / N, or 8 + gradient + 16 / N with the mean.
-constexpr int kBatch = 4;  // replicas of one vector loaded together; two batches are in flight
+constexpr int kChunk = 8;      // replicas of one vector whose parameters are loaded together
+constexpr int kGradChunk = 4;  // replicas whose bf16 gradients are loaded together for the mean (fp32: half)
 
 template <typename GradT, bool kConv, bool kMean>
 __device__ void range_scalar_shared(const TensorDesc& td, long long begin, long long end, const StepScalars& s,
@@ -326,109 +327,100 @@ __device__ __forceinline__ void tile_vector_shared(const TensorDesc& td, long lo
   float* const M = td.exp_avg + off;
   float* const V = td.exp_avg_sq + off;
   const GradT* const Gp = static_cast<const GradT*>(td.grad) + off;
-  const long long ps = td.param_stride;
+  const long long ps = td.param_stride, gs = td.grad_stride;
 
-  int idx[kTileVecs];
-  bool ok[kTileVecs];
+  // One float4 vector at a time: all loads of the vector (up to kChunk replicas of theta, the gradient(s),
+  // both moments) are issued together, so little register state is needed and three CTAs fit on an SM.
 #pragma unroll
   for (int k = 0; k < kTileVecs; ++k) {
     const int j = k * kThreads + threadIdx.x;
-    idx[k] = j * 4;
-    ok[k] = kFull || j < nvec;
-  }
+    if (!kFull && j >= nvec) continue;
+    const int at = j * 4;
 
-  using Batch = float4[kBatch];
-  auto load_batch = [&](Batch& buf, int r0, int at, bool valid) {
+    // Parameters of up to kChunk replicas and both moments are requested first; the gradient (for the
+    // replica mean: N loads in groups of kGradChunk, summed in fp64) is consumed while they are in flight.
+    float4 th[kChunk];
 #pragma unroll
-    for (int j = 0; j < kBatch; ++j)
-      buf[j] = (valid && r0 + j < n) ? __ldcs(reinterpret_cast<const float4*>(P + (r0 + j) * ps + at))
-                                     : make_float4(0.f, 0.f, 0.f, 0.f);
-  };
-
-  // The first parameters are requested before the gradient and the moments are consumed.
-  Batch a, b;
-  load_batch(a, 0, idx[0], ok[0]);
-
-  // Step direction u = m' / (sqrt(v')/sqrt(bc2) + eps), once per element for all replicas.
-  float u[kTileVecs][4];
-  if constexpr (kMean) {
-    mean_gradient<GradT>(Gp, td.grad_stride, idx, ok, n, s.inv_n, u);
-  } else {
+    for (int q = 0; q < kChunk; ++q)
+      th[q] = q < n ? __ldcs(reinterpret_cast<const float4*>(P + q * ps + at)) : make_float4(0.f, 0.f, 0.f, 0.f);
+    const float4 m4 = __ldcs(reinterpret_cast<const float4*>(M + at));
+    const float4 v4 = __ldcs(reinterpret_cast<const float4*>(V + at));
+    float g[4];
+    if constexpr (kMean) {
+      double acc[4] = {0.0, 0.0, 0.0, 0.0};
+      constexpr int kG = sizeof(typename GradRaw<GradT>::type) == 16 ? kGradChunk / 2 : kGradChunk;
+      for (int r0 = 0; r0 < n; r0 += kG) {
+        typename GradRaw<GradT>::type raw[kG];
 #pragma unroll
-    for (int k = 0; k < kTileVecs; ++k) {
-      if (ok[k]) {
-        unpack(load_raw(Gp + idx[k]), u[k]);
-      } else {
+        for (int q = 0; q < kG; ++q)
+          if (r0 + q < n) raw[q] = load_raw(Gp + (r0 + q) * gs + at);
 #pragma unroll
-        for (int q = 0; q < 4; ++q) u[k][q] = 0.f;
-      }
-    }
-  }
+        for (int q = 0; q < kG; ++q) {
+          if (r0 + q < n) {
+            float gr[4];
+            unpack(raw[q], gr);
 #pragma unroll
-  for (int k = 0; k < kTileVecs; ++k) {
-    float4 m4 = make_float4(0.f, 0.f, 0.f, 0.f), v4 = m4;
-    if (ok[k]) {
-      m4 = __ldcs(reinterpret_cast<const float4*>(M + idx[k]));
-      v4 = __ldcs(reinterpret_cast<const float4*>(V + idx[k]));
-    }
-    float m[4] = {m4.x, m4.y, m4.z, m4.w};
-    float v[4] = {v4.x, v4.y, v4.z, v4.w};
-#pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      const float g = u[k][q];
-      m[q] = fmaf(c.one_minus_beta1, g - m[q], m[q]);
-      v[q] = fmaf(c.one_minus_beta2, fmaf(g, g, -v[q]), v[q]);
-      u[k][q] = m[q] / fmaf(sqrtf(v[q]), c.rsqrt_bc2, c.eps);
-    }
-    if (ok[k]) {
-      __stcs(reinterpret_cast<float4*>(M + idx[k]), make_float4(m[0], m[1], m[2], m[3]));
-      __stcs(reinterpret_cast<float4*>(V + idx[k]), make_float4(v[0], v[1], v[2], v[3]));
-    }
-  }
-
-  // Replicas: per vector, batches of kBatch replicas, the next batch in flight while one is updated.
-#pragma unroll
-  for (int k = 0; k < kTileVecs; ++k) {
-    double sum[4] = {0.0, 0.0, 0.0, 0.0};
-    auto update_batch = [&](Batch& buf, int r0) {
-#pragma unroll
-      for (int j = 0; j < kBatch; ++j) {
-        const int r = r0 + j;
-        if (r < n) {
-          const float lr_wd = s.lr_wd[grp][r];
-          const float step = s.step[grp][r];
-          float th[4] = {buf[j].x, buf[j].y, buf[j].z, buf[j].w};
-#pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            th[q] = fmaf(-step, u[k][q], fmaf(-lr_wd, th[q], th[q]));
-            bad |= not_finite(th[q]);
-          }
-          if (kConv) {
-#pragma unroll
-            for (int q = 0; q < 4; ++q) sum[q] += (double)th[q];
-          } else if (ok[k]) {
-            __stcs(reinterpret_cast<float4*>(P + r * ps + idx[k]), make_float4(th[0], th[1], th[2], th[3]));
+            for (int e = 0; e < 4; ++e) acc[e] += (double)gr[e];
           }
         }
       }
-    };
-    if (k > 0) load_batch(a, 0, idx[k], ok[k]);
-    for (int r0 = 0; r0 < n; r0 += 2 * kBatch) {
-      if (r0 + kBatch < n) load_batch(b, r0 + kBatch, idx[k], ok[k]);
-      update_batch(a, r0);
-      if (r0 + 2 * kBatch < n) load_batch(a, r0 + 2 * kBatch, idx[k], ok[k]);
-      if (r0 + kBatch < n) update_batch(b, r0 + kBatch);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) g[q] = (float)(acc[q] * s.inv_n);
     }
-    if (kConv && ok[k]) {
+    if constexpr (!kMean) unpack(load_raw(Gp + at), g);
+
+    // Step direction u = m' / (sqrt(v')/sqrt(bc2) + eps), once per element for all replicas.
+    float m[4] = {m4.x, m4.y, m4.z, m4.w};
+    float v[4] = {v4.x, v4.y, v4.z, v4.w};
+    float u[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      m[q] = fmaf(c.one_minus_beta1, g[q] - m[q], m[q]);
+      v[q] = fmaf(c.one_minus_beta2, fmaf(g[q], g[q], -v[q]), v[q]);
+      u[q] = m[q] / fmaf(sqrtf(v[q]), c.rsqrt_bc2, c.eps);
+    }
+    __stcs(reinterpret_cast<float4*>(M + at), make_float4(m[0], m[1], m[2], m[3]));
+    __stcs(reinterpret_cast<float4*>(V + at), make_float4(v[0], v[1], v[2], v[3]));
+
+    double sum[4] = {0.0, 0.0, 0.0, 0.0};
+    for (int r0 = 0; r0 < n; r0 += kChunk) {
+      if (r0 > 0) {
+#pragma unroll
+        for (int q = 0; q < kChunk; ++q)
+          th[q] = r0 + q < n ? __ldcs(reinterpret_cast<const float4*>(P + (r0 + q) * ps + at))
+                             : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+#pragma unroll
+      for (int q = 0; q < kChunk; ++q) {
+        const int r = r0 + q;
+        if (r < n) {
+          const float lr_wd = s.lr_wd[grp][r];
+          const float step = s.step[grp][r];
+          float t4[4] = {th[q].x, th[q].y, th[q].z, th[q].w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            t4[e] = fmaf(-step, u[e], fmaf(-lr_wd, t4[e], t4[e]));
+            bad |= not_finite(t4[e]);
+          }
+          if (kConv) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) sum[e] += (double)t4[e];
+          } else {
+            __stcs(reinterpret_cast<float4*>(P + r * ps + at), make_float4(t4[0], t4[1], t4[2], t4[3]));
+          }
+        }
+      }
+    }
+    if (kConv) {
       const float4 mean = make_float4((float)(sum[0] * s.inv_n), (float)(sum[1] * s.inv_n),
                                       (float)(sum[2] * s.inv_n), (float)(sum[3] * s.inv_n));
-      for (int rr = 0; rr < n; ++rr) __stcs(reinterpret_cast<float4*>(P + rr * ps + idx[k]), mean);
+      for (int rr = 0; rr < n; ++rr) __stcs(reinterpret_cast<float4*>(P + rr * ps + at), mean);
     }
   }
 }
 
 template <typename GradT, bool kConv, bool kMean>
-__global__ void __launch_bounds__(kThreads, 2)
+__global__ void __launch_bounds__(kThreads, 3)
 fanout_shared_kernel(const __grid_constant__ LaunchPlan plan, const __grid_constant__ StepScalars s) {
   const AdamConsts c{s.one_minus_beta1, s.one_minus_beta2, s.rsqrt_bc2, s.eps};
   bool bad = false;
