@@ -220,16 +220,45 @@ def run_ours(args):
     losses = [list(R.step_losses(w, i % w.total_steps)) for i in range(w.total_steps)]
     state = {"i": 0}
 
+    d_losses = torch.tensor(np.array(losses), dtype=torch.float64, device=f"cuda:{local}")
+    steps_per_call = 1
+    graph = None
+
     def one_step():
-        if B.hdet_step(h, losses[state["i"] % w.total_steps], stream.cuda_stream):
-            B.hdet_autolr_update(h)
-        state["i"] += 1
+        """One update (or, with --stepping graph, one recorded round of T updates)."""
+        k = state["i"] % w.total_steps
+        if args.stepping == "host":
+            if B.hdet_step(h, losses[k], stream.cuda_stream):
+                B.hdet_autolr_update(h)
+        elif args.stepping == "device":
+            B.hdet_step_device(h, d_losses[k], stream.cuda_stream)
+        else:
+            graph.replay()
+        state["i"] += steps_per_call
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
+    if args.stepping == "graph":
+        # One round of T device-resident updates is run directly (uploads the state), then recorded once;
+        # every call of one_step() replays the recorded round.
+        T = w.sync_interval
+        if args.steps % T:
+            raise SystemExit(f"--stepping graph needs --steps to be a multiple of the sync interval {T}")
+        for k in range(T):
+            B.hdet_step_device(h, d_losses[k % w.total_steps], stream.cuda_stream)
+        torch.cuda.synchronize()
+        side = torch.cuda.Stream()
+        graph = torch.cuda.CUDAGraph()
+        before = B.hdet_kernel_launches(h)
+        with torch.cuda.graph(graph, stream=side):
+            for k in range(T):
+                B.hdet_step_device(h, d_losses[k % w.total_steps], torch.cuda.current_stream().cuda_stream)
+        launches_per_call = B.hdet_kernel_launches(h) - before
+        steps_per_call = T
+    n_calls = args.steps // steps_per_call
     for _ in range(max(args.warmup, 3)):
         one_step()
     barrier()
@@ -237,17 +266,19 @@ def run_ours(args):
     # ---- device-timed region: inputs resident in HBM -------------------------------------------------
     sampler = ClockSampler(local) if rank == 0 else None
     launches0 = B.hdet_kernel_launches(h)
-    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(n_calls + 1)]
     barrier()
     ev[0].record(stream)
-    for k in range(args.steps):
+    for k in range(n_calls):
         one_step()
         ev[k + 1].record(stream)
     barrier()
     clocks = sampler.stop() if sampler else None
     launches = B.hdet_kernel_launches(h) - launches0
+    if args.stepping == "graph":
+        launches = launches_per_call * n_calls          # replays launch the recorded kernels without calling the library
     total_ms = ev[0].elapsed_time(ev[-1])
-    per_step_ms = [ev[k].elapsed_time(ev[k + 1]) for k in range(args.steps)]
+    per_step_ms = [ev[k].elapsed_time(ev[k + 1]) / steps_per_call for k in range(n_calls)]
     ms_per_step = max_over_ranks(total_ms, world, f"cuda:{local}") / args.steps
     value = whole_job_value(n * P, world, ms_per_step)
 
@@ -261,7 +292,11 @@ def run_ours(args):
     def e2e_step():
         for r in range(n_grad_copies):
             (arena.grad if args.shared_grad else arena.grad[r]).copy_(host_grad, non_blocking=True)
-        one_step()
+        if args.stepping == "host":
+            one_step()
+        else:                                               # per step, so that every step sees its own gradients
+            B.hdet_step_device(h, d_losses[state["i"] % w.total_steps], stream.cuda_stream)
+            state["i"] += 1
         st = B.hdet_get_state(h, raise_on_nonfinite=False)   # reads the device status word back (synchronises)
         return st.device_status
 
@@ -315,7 +350,8 @@ def run_ours(args):
 
     bpe = bytes_per_element(w, args.shared_grad, args.shared_state)
     peak, peak_src = measured_peaks()
-    launch_ms = statistics.mean(per_step_ms) / max(1, launches // args.steps)
+    # mean duration of one fan-out launch: a step is one fan-out launch (device stepping adds one-warp scalar kernels)
+    launch_ms = statistics.mean(per_step_ms)
     achieved = bpe * n * P / (launch_ms * 1e-3) / 1e9
     traffic, traffic_src = args.traffic_bytes, "command line" if args.traffic_bytes else None
     plain_mode = not (args.shared_grad or args.shared_state or args.grad_mode == "mean")
@@ -331,7 +367,7 @@ def run_ours(args):
         "config": {
             "workload": w.name, "n_replicas": n, "params_per_replica": P, "n_tensors": len(w.tensors),
             "optimizer": "adamw" if w.optimizer == W.OPT_ADAMW else "sgd", "sync_interval": w.sync_interval,
-            "alpha_lr": w.alpha_lr, "grad_mode": args.grad_mode, "shared_grad": args.shared_grad,
+            "alpha_lr": w.alpha_lr, "stepping": args.stepping, "grad_mode": args.grad_mode, "shared_grad": args.shared_grad,
             "shared_moments": args.shared_state, "resident_gb": arena.resident_bytes() / 1e9,
             "l2_policy": "inputs larger than L2 (no flush)", "parallelism": f"{world} independent replicas of the job",
             "note": note,
@@ -389,6 +425,9 @@ def main():
     ap.add_argument("--workload", default="config4", choices=sorted(W.ALL_CONFIGS))
     ap.add_argument("--sync-interval", type=int, default=None,
                     help="override the workload's T (e.g. 1 to profile the fused update+converge kernel on a small list)")
+    ap.add_argument("--stepping", default="host", choices=["host", "device", "graph"],
+                    help="host: hdet_step (+ hdet_autolr_update); device: hdet_step_device with device losses; "
+                         "graph: a recorded round of hdet_step_device calls replayed")
     ap.add_argument("--grad-mode", default="as_given", choices=["as_given", "mean"],
                     help="mean: every replica steps with the on-device replica mean of the gradients")
     ap.add_argument("--shared-grad", action="store_true", help="one gradient for all replicas (grad_stride 0)")

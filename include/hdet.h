@@ -61,7 +61,7 @@ typedef enum {
 } hdet_status;
 
 enum { HDET_OPT_SGD = 0, HDET_OPT_ADAMW = 1 };
-enum { HDET_DTYPE_F32 = 0, HDET_DTYPE_BF16 = 1 };
+enum { HDET_DTYPE_F32 = 0, HDET_DTYPE_BF16 = 1, HDET_DTYPE_F64 = 2 /* losses only */ };
 enum { HDET_GRAD_AS_GIVEN = 0, HDET_GRAD_REPLICA_MEAN = 1 };
 enum { HDET_SCHED_CONSTANT = 0, HDET_SCHED_ONECYCLE_COS = 1, HDET_SCHED_ONECYCLE_LINEAR = 2 };
 
@@ -195,6 +195,30 @@ HDET_API int hdet_set_schedule(hdet_handle h, const hdet_schedule* sched);
 HDET_API int hdet_step(hdet_handle h, const double* step_losses, void* stream, int32_t* did_converge);
 
 /*
+ * hdet_step_device -- hdet_step and, at the end of a round, hdet_autolr_update, with Algorithm 1's
+ * scalar state kept on the device: nothing is computed on the host, nothing is copied, and the
+ * losses are read from DEVICE memory (d_step_losses: N values of loss_dtype HDET_DTYPE_F32 or
+ * HDET_DTYPE_F64, or NULL), so a training loop never has to wait for a loss to reach the host.
+ * Per call: a one-warp fp64 kernel evaluates the schedule, Eq. 1 and the permutations of Eq. 9 into
+ * the launch scalars and accumulates the losses; the fan-out kernel (fused with Eq. 3 on the last
+ * update of a round) reads those scalars from device memory; after a round's last update a second
+ * one-warp kernel latches the mean losses and, if auto-LR is on and t >= S_warm, runs Eq. 4 - Eq. 9
+ * (softmax and sums by warp shuffles, one lane per replica).  The same double-precision code as the
+ * host path is compiled for the device, so scalars agree with it to rounding of the math library.
+ * Which kernels a call launches depends only on the step count, so a whole round of T calls can be
+ * recorded once and replayed.  *did_converge as for hdet_step (may be NULL).
+ * The first call after hdet_create / hdet_set_state copies the host state to the device with a
+ * blocking copy; from then on the device copy is authoritative: hdet_get_state reads it back
+ * (blocking) and refreshes the host copy, hdet_set_state returns the handle to host stepping, and
+ * hdet_step / hdet_autolr_update return HDET_ERR_STATE in between.  If steps were replayed without
+ * calling this function, call hdet_get_state before the next direct call so that the host knows the
+ * step count again.
+ * Errors: INVALID_ARG, STATE (no schedule), UNSUPPORTED (handle without tensors), CUDA.
+ */
+HDET_API int hdet_step_device(hdet_handle h, const void* d_step_losses, int32_t loss_dtype, void* stream,
+                              int32_t* did_converge);
+
+/*
  * hdet_converge -- Eq. 3 on its own: theta_r <- (1/N) sum_r' theta_r' for every tensor.
  * Does not touch the step count, the moments or the loss accumulator.
  * Errors: INVALID_ARG, CUDA.
@@ -225,7 +249,9 @@ HDET_API int hdet_get_state(hdet_handle h, hdet_state* out);
 /*
  * hdet_set_state -- restores step, n_acc, fired, round_ended, ctrl_base, velocity, the
  * permutations, loss_acc and loss_round from *in (resume); the other fields are
- * recomputed.  Clears the device status word.
+ * recomputed.  Clears the device status word.  Waits for the device to become idle (earlier
+ * device-resident steps must not outlive the state they read) and returns the handle to host
+ * stepping.
  * Errors: INVALID_ARG (NULL, negative step, an array that is not a permutation).
  */
 HDET_API int hdet_set_state(hdet_handle h, const hdet_state* in);

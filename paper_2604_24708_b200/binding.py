@@ -21,7 +21,7 @@ HDET_ERR_CUDA = 5
 HDET_ERR_NONFINITE = 6
 
 HDET_OPT_SGD, HDET_OPT_ADAMW = 0, 1
-HDET_DTYPE_F32, HDET_DTYPE_BF16 = 0, 1
+HDET_DTYPE_F32, HDET_DTYPE_BF16, HDET_DTYPE_F64 = 0, 1, 2
 HDET_GRAD_AS_GIVEN, HDET_GRAD_REPLICA_MEAN = 0, 1
 HDET_SCHED_CONSTANT, HDET_SCHED_ONECYCLE_COS, HDET_SCHED_ONECYCLE_LINEAR = 0, 1, 2
 
@@ -89,6 +89,8 @@ def _load() -> C.CDLL:
     lib.hdet_create.argtypes = [C.POINTER(hdet_config), C.POINTER(hdet_tensor), C.c_int64, C.POINTER(H)]
     lib.hdet_set_schedule.argtypes = [H, C.POINTER(hdet_schedule)]
     lib.hdet_step.argtypes = [H, C.POINTER(C.c_double), C.c_void_p, C.POINTER(C.c_int32)]
+    lib.hdet_step_device.argtypes = [H, C.c_void_p, C.c_int32, C.c_void_p, C.POINTER(C.c_int32)]
+    lib.hdet_step_device.restype = C.c_int
     lib.hdet_converge.argtypes = [H, C.c_void_p]
     lib.hdet_autolr_update.argtypes = [H, C.POINTER(C.c_double), C.c_void_p]
     lib.hdet_get_state.argtypes = [H, C.POINTER(hdet_state)]
@@ -182,6 +184,20 @@ def hdet_step(h, step_losses: Optional[Sequence[float]] = None, stream: int = 0)
     """Runs one update; returns True when it ended a round (the replicas were averaged)."""
     flag = C.c_int32(0)
     _check(_lib.hdet_step(h, _doubles(step_losses), C.c_void_p(stream), C.byref(flag)), h)
+    return bool(flag.value)
+
+
+def hdet_step_device(h, d_step_losses=None, stream: int = 0) -> bool:
+    """One device-resident update; ``d_step_losses`` is a CUDA tensor of N float32 or float64 losses (or None)."""
+    flag = C.c_int32(0)
+    ptr, dtype = None, HDET_DTYPE_F32
+    if d_step_losses is not None:
+        import torch
+        if not d_step_losses.is_cuda or not d_step_losses.is_contiguous():
+            raise ValueError("d_step_losses must be a contiguous CUDA tensor")
+        dtype = {torch.float32: HDET_DTYPE_F32, torch.float64: HDET_DTYPE_F64}[d_step_losses.dtype]
+        ptr = C.c_void_p(d_step_losses.data_ptr())
+    _check(_lib.hdet_step_device(h, ptr, dtype, C.c_void_p(stream), C.byref(flag)), h)
     return bool(flag.value)
 
 

@@ -7,6 +7,7 @@
 #include <string>
 #include <vector>
 
+#include "hdet_device_state.cuh"
 #include "hdet_internal.h"
 #include "hdet_kernels.cuh"
 #include "hdet_scalars.h"
@@ -43,6 +44,8 @@ struct hdet_ctx {
   TensorDesc* d_tensors = nullptr;
   Tile* d_tiles = nullptr;
   unsigned* d_status = nullptr;
+  DevState* d_state = nullptr;   // device-resident scalar state (used by hdet_step_device)
+  bool device_mode = false;      // the device copy of the state is the authoritative one
   int n_tiles = 0;
   int grid_fanout = 0;
   int grid_converge = 0;
@@ -85,7 +88,8 @@ void free_device(hdet_ctx* h) {
   if (h->d_tensors) cudaFree(h->d_tensors);
   if (h->d_tiles) cudaFree(h->d_tiles);
   if (h->d_status) cudaFree(h->d_status);
-  h->d_tensors = nullptr; h->d_tiles = nullptr; h->d_status = nullptr;
+  if (h->d_state) cudaFree(h->d_state);
+  h->d_tensors = nullptr; h->d_tiles = nullptr; h->d_status = nullptr; h->d_state = nullptr;
 }
 
 // Rates and weight decays for the update at 0-based index h->step.
@@ -110,6 +114,69 @@ bool is_permutation(const int32_t* p, int n) {
     seen[p[r]] = true;
   }
   return true;
+}
+
+// Host fields -> public state block (no device access).
+void export_state(const hdet_ctx* h, hdet_state* out) {
+  std::memset(out, 0, sizeof *out);
+  out->step = h->step;
+  out->n_acc = h->n_acc;
+  out->fired = h->fired;
+  out->round_ended = h->round_ended;
+  std::memcpy(out->base, h->base, sizeof h->base);
+  std::memcpy(out->ctrl_base, h->ctrl_base, sizeof h->ctrl_base);
+  std::memcpy(out->velocity, h->velocity, sizeof h->velocity);
+  std::memcpy(out->delta, h->delta, sizeof h->delta);
+  std::memcpy(out->lr, h->lr, sizeof h->lr);
+  std::memcpy(out->wd, h->wd, sizeof h->wd);
+  std::memcpy(out->perm_lr, h->perm_lr, sizeof h->perm_lr);
+  std::memcpy(out->perm_wd, h->perm_wd, sizeof h->perm_wd);
+  std::memcpy(out->weights, h->weights, sizeof h->weights);
+  std::memcpy(out->loss_acc, h->loss_acc, sizeof h->loss_acc);
+  std::memcpy(out->loss_round, h->loss_round, sizeof h->loss_round);
+  out->gamma = h->has_schedule ? decay_gamma(h->sched.f_div, h->sched.f_final, h->sched.total_steps,
+                                             h->sched.warmup_steps, h->cfg.sync_interval)
+                               : 0.0;
+}
+
+// Public state block -> host fields (everything, including the tables of the last update).
+void import_state(hdet_ctx* h, const hdet_state* in) {
+  h->step = in->step;
+  h->n_acc = in->n_acc;
+  h->fired = in->fired != 0;
+  h->round_ended = in->round_ended != 0;
+  std::memcpy(h->base, in->base, sizeof h->base);
+  std::memcpy(h->ctrl_base, in->ctrl_base, sizeof h->ctrl_base);
+  std::memcpy(h->velocity, in->velocity, sizeof h->velocity);
+  std::memcpy(h->delta, in->delta, sizeof h->delta);
+  std::memcpy(h->lr, in->lr, sizeof h->lr);
+  std::memcpy(h->wd, in->wd, sizeof h->wd);
+  std::memcpy(h->perm_lr, in->perm_lr, sizeof h->perm_lr);
+  std::memcpy(h->perm_wd, in->perm_wd, sizeof h->perm_wd);
+  std::memcpy(h->weights, in->weights, sizeof h->weights);
+  std::memcpy(h->loss_acc, in->loss_acc, sizeof h->loss_acc);
+  std::memcpy(h->loss_round, in->loss_round, sizeof h->loss_round);
+}
+
+DevConst device_constants(const hdet_ctx* h) {
+  DevConst c{};
+  c.n = h->cfg.n_replicas;
+  c.n_groups = h->cfg.n_groups;
+  c.adam = h->cfg.optimizer == HDET_OPT_ADAMW;
+  c.kind = h->sched.kind;
+  c.autolr = h->sched.autolr;
+  c.reshuffle = h->cfg.reshuffle;
+  c.total_steps = h->sched.total_steps;
+  c.warmup_steps = h->sched.warmup_steps;
+  c.sync_interval = h->cfg.sync_interval;
+  c.beta1 = h->cfg.beta1; c.beta2 = h->cfg.beta2; c.eps = h->cfg.eps;
+  c.alpha_lr = h->cfg.alpha_lr; c.alpha_wd = h->cfg.alpha_wd;
+  c.pct_start = h->sched.pct_start; c.div_factor = h->sched.div_factor; c.final_div_factor = h->sched.final_div_factor;
+  c.ctrl_beta = h->sched.beta; c.sigma = h->sched.sigma; c.lambda = h->sched.lambda;
+  c.f_div = h->sched.f_div; c.f_final = h->sched.f_final;
+  for (int g = 0; g < HDET_MAX_GROUPS; ++g) { c.max_lr[g] = h->max_lr[g]; c.weight_decay[g] = h->weight_decay[g]; }
+  c.seed = h->cfg.seed;
+  return c;
 }
 
 }  // namespace
@@ -215,6 +282,7 @@ int hdet_create(const hdet_config* cfg, const hdet_tensor* tensors, int64_t n_te
     if (e == cudaSuccess) e = cudaMalloc(&h->d_tensors, descs.size() * sizeof(TensorDesc));
     if (e == cudaSuccess) e = cudaMalloc(&h->d_tiles, tiles.size() * sizeof(Tile));
     if (e == cudaSuccess) e = cudaMalloc(&h->d_status, sizeof(unsigned));
+    if (e == cudaSuccess) e = cudaMalloc(&h->d_state, sizeof(DevState));
     if (e == cudaSuccess) e = cudaMemcpy(h->d_tensors, descs.data(), descs.size() * sizeof(TensorDesc), cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemcpy(h->d_tiles, tiles.data(), tiles.size() * sizeof(Tile), cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemset(h->d_status, 0, sizeof(unsigned));
@@ -272,6 +340,8 @@ int hdet_step(hdet_handle h, const double* step_losses, void* stream, int32_t* d
   if (!h) return HDET_ERR_INVALID_ARG;
   if (did_converge) *did_converge = 0;
   if (!h->has_schedule) return fail(h, HDET_ERR_STATE, "hdet_step: call hdet_set_schedule first");
+  if (h->device_mode)
+    return fail(h, HDET_ERR_STATE, "hdet_step: the handle steps on the device (hdet_step_device); hdet_set_state returns it to host stepping");
   const int n = h->cfg.n_replicas, G = h->cfg.n_groups;
   compute_tables(h);
   const int64_t t = h->step + 1;
@@ -301,7 +371,7 @@ int hdet_step(hdet_handle h, const double* step_losses, void* stream, int32_t* d
     if (scope.err != cudaSuccess) return fail_cuda(h, "hdet_step", scope.err);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const bool fuse = ends_round && h->cfg.fuse_converge;
-    LaunchPlan plan{h->d_tensors, h->d_tiles, h->n_tiles, h->grid_fanout, h->d_status};
+    LaunchPlan plan{h->d_tensors, h->d_tiles, h->n_tiles, h->grid_fanout, h->d_status, nullptr};
     cudaError_t e = launch_fanout(h->cfg.optimizer, h->cfg.grad_dtype, fuse, h->cfg.grad_mode == HDET_GRAD_REPLICA_MEAN,
                                   h->shared_state, plan, s, st);
     if (e != cudaSuccess) return fail_cuda(h, "hdet_step: fan-out launch", e);
@@ -331,12 +401,66 @@ int hdet_step(hdet_handle h, const double* step_losses, void* stream, int32_t* d
   return HDET_OK;
 }
 
+int hdet_step_device(hdet_handle h, const void* d_step_losses, int32_t loss_dtype, void* stream, int32_t* did_converge) {
+  if (!h) return HDET_ERR_INVALID_ARG;
+  if (did_converge) *did_converge = 0;
+  if (!h->has_schedule) return fail(h, HDET_ERR_STATE, "hdet_step_device: call hdet_set_schedule first");
+  if (h->n_tiles == 0 || !h->d_state)
+    return fail(h, HDET_ERR_UNSUPPORTED, "hdet_step_device: the handle has no tensors, hence no device state");
+  if (d_step_losses && loss_dtype != HDET_DTYPE_F32 && loss_dtype != HDET_DTYPE_F64)
+    return fail(h, HDET_ERR_INVALID_ARG, "hdet_step_device: losses must be fp32 or fp64");
+  DeviceScope scope(h->cfg.device);
+  if (scope.err != cudaSuccess) return fail_cuda(h, "hdet_step_device", scope.err);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (!h->device_mode) {
+    // First device-resident step: the host state becomes the device state (one blocking copy).
+    hdet_state snapshot;
+    export_state(h, &snapshot);
+    cudaError_t e = cudaMemcpy(&h->d_state->st, &snapshot, sizeof snapshot, cudaMemcpyHostToDevice);
+    if (e != cudaSuccess) return fail_cuda(h, "hdet_step_device: state upload", e);
+    h->device_mode = true;
+  }
+  const int n = h->cfg.n_replicas;
+  const int64_t t = h->step + 1;
+  const bool ends_round = (t % h->cfg.sync_interval) == 0;
+  const DevConst c = device_constants(h);
+  cudaError_t e = launch_device_scalars(h->d_state, c, d_step_losses, loss_dtype == HDET_DTYPE_F64, st);
+  if (e != cudaSuccess) return fail_cuda(h, "hdet_step_device: scalar kernel launch", e);
+  ++h->launches;
+  const bool fuse = ends_round && h->cfg.fuse_converge;
+  LaunchPlan plan{h->d_tensors, h->d_tiles, h->n_tiles, h->grid_fanout, h->d_status, &h->d_state->scal};
+  const StepScalars unused{};
+  e = launch_fanout(h->cfg.optimizer, h->cfg.grad_dtype, fuse, h->cfg.grad_mode == HDET_GRAD_REPLICA_MEAN,
+                    h->shared_state, plan, unused, st);
+  if (e != cudaSuccess) return fail_cuda(h, "hdet_step_device: fan-out launch", e);
+  ++h->launches;
+  if (ends_round && !fuse) {
+    plan.grid = h->grid_converge;
+    e = launch_converge(plan, n, st);
+    if (e != cudaSuccess) return fail_cuda(h, "hdet_step_device: converge launch", e);
+    ++h->launches;
+  }
+  // Host shadow of what is known without reading the device: the step count and the round position.
+  h->step = t;
+  ++h->n_acc;
+  h->round_ended = false;
+  if (ends_round) {
+    e = launch_device_round_end(h->d_state, c, st);
+    if (e != cudaSuccess) return fail_cuda(h, "hdet_step_device: controller launch", e);
+    ++h->launches;
+    h->n_acc = 0;
+    if (h->sched.autolr && t >= h->sched.warmup_steps) h->fired = true;
+    if (did_converge) *did_converge = 1;
+  }
+  return HDET_OK;
+}
+
 int hdet_converge(hdet_handle h, void* stream) {
   if (!h) return HDET_ERR_INVALID_ARG;
   if (h->n_tiles == 0) return HDET_OK;
   DeviceScope scope(h->cfg.device);
   if (scope.err != cudaSuccess) return fail_cuda(h, "hdet_converge", scope.err);
-  LaunchPlan plan{h->d_tensors, h->d_tiles, h->n_tiles, h->grid_converge, h->d_status};
+  LaunchPlan plan{h->d_tensors, h->d_tiles, h->n_tiles, h->grid_converge, h->d_status, nullptr};
   cudaError_t e = launch_converge(plan, h->cfg.n_replicas, static_cast<cudaStream_t>(stream));
   if (e != cudaSuccess) return fail_cuda(h, "hdet_converge: launch", e);
   ++h->launches;
@@ -346,6 +470,8 @@ int hdet_converge(hdet_handle h, void* stream) {
 int hdet_autolr_update(hdet_handle h, const double* round_losses, void* /*stream*/) {
   if (!h) return HDET_ERR_INVALID_ARG;
   if (!h->has_schedule) return fail(h, HDET_ERR_STATE, "hdet_autolr_update: call hdet_set_schedule first");
+  if (h->device_mode)
+    return fail(h, HDET_ERR_STATE, "hdet_autolr_update: with hdet_step_device the controller already runs on the device");
   if (!h->round_ended)
     return fail(h, HDET_ERR_STATE, "hdet_autolr_update: the last hdet_step did not end a round (or the update already ran)");
   h->round_ended = false;
@@ -387,25 +513,16 @@ int hdet_autolr_update(hdet_handle h, const double* round_losses, void* /*stream
 int hdet_get_state(hdet_handle h, hdet_state* out) {
   if (!h) return HDET_ERR_INVALID_ARG;
   if (!out) return fail(h, HDET_ERR_INVALID_ARG, "hdet_get_state: out is NULL");
-  std::memset(out, 0, sizeof *out);
-  out->step = h->step;
-  out->n_acc = h->n_acc;
-  out->fired = h->fired;
-  out->round_ended = h->round_ended;
-  std::memcpy(out->base, h->base, sizeof h->base);
-  std::memcpy(out->ctrl_base, h->ctrl_base, sizeof h->ctrl_base);
-  std::memcpy(out->velocity, h->velocity, sizeof h->velocity);
-  std::memcpy(out->delta, h->delta, sizeof h->delta);
-  std::memcpy(out->lr, h->lr, sizeof h->lr);
-  std::memcpy(out->wd, h->wd, sizeof h->wd);
-  std::memcpy(out->perm_lr, h->perm_lr, sizeof h->perm_lr);
-  std::memcpy(out->perm_wd, h->perm_wd, sizeof h->perm_wd);
-  std::memcpy(out->weights, h->weights, sizeof h->weights);
-  std::memcpy(out->loss_acc, h->loss_acc, sizeof h->loss_acc);
-  std::memcpy(out->loss_round, h->loss_round, sizeof h->loss_round);
-  out->gamma = h->has_schedule ? decay_gamma(h->sched.f_div, h->sched.f_final, h->sched.total_steps,
-                                             h->sched.warmup_steps, h->cfg.sync_interval)
-                               : 0.0;
+  if (h->device_mode) {
+    // The device copy is authoritative: read it back (blocking) and refresh the host fields from it.
+    DeviceScope scope(h->cfg.device);
+    cudaError_t e = scope.err;
+    hdet_state dev;
+    if (e == cudaSuccess) e = cudaMemcpy(&dev, &h->d_state->st, sizeof dev, cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return fail_cuda(h, "hdet_get_state: state read-back", e);
+    import_state(h, &dev);
+  }
+  export_state(h, out);
   if (h->d_status) {
     DeviceScope scope(h->cfg.device);
     cudaError_t e = scope.err;
@@ -439,9 +556,11 @@ int hdet_set_state(hdet_handle h, const hdet_state* in) {
   }
   std::memcpy(h->loss_acc, in->loss_acc, sizeof h->loss_acc);
   std::memcpy(h->loss_round, in->loss_round, sizeof h->loss_round);
+  h->device_mode = false;   // the host copy is authoritative again; hdet_step_device uploads it anew
   if (h->d_status) {
     DeviceScope scope(h->cfg.device);
     cudaError_t e = scope.err;
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();   // earlier device-resident steps must not outlive the state they use
     if (e == cudaSuccess) e = cudaMemset(h->d_status, 0, sizeof(unsigned));
     if (e != cudaSuccess) return fail_cuda(h, "hdet_set_state", e);
   }
@@ -450,7 +569,7 @@ int hdet_set_state(hdet_handle h, const hdet_state* in) {
 
 int hdet_destroy(hdet_handle h) {
   if (!h) return HDET_OK;
-  if (h->d_tensors || h->d_tiles || h->d_status) {
+  if (h->d_tensors || h->d_tiles || h->d_status || h->d_state) {
     DeviceScope scope(h->cfg.device);
     free_device(h);
   }

@@ -247,9 +247,36 @@ __device__ __forceinline__ void tile_vector(const TensorDesc& td, long long off,
   }
 }
 
+// The launch scalars are staged in shared memory once per CTA, from the kernel parameter (host stepping)
+// or from the device-resident copy (device stepping); the update loops then read them with broadcast
+// shared-memory loads.  Selecting between the two sources by pointer instead costs 7 % of the kernel's
+// bandwidth: the by-value parameter is then no longer read through the constant bank.
+__device__ __forceinline__ void stage_scalars(StepScalars& sh, const StepScalars& s_param, const StepScalars* s_dev) {
+  static_assert(HDET_MAX_GROUPS * HDET_MAX_REPLICAS == kThreads, "one (group, replica) pair per thread");
+  const int g = threadIdx.x / HDET_MAX_REPLICAS, r = threadIdx.x % HDET_MAX_REPLICAS;
+  if (s_dev) {
+    sh.lr_wd[g][r] = s_dev->lr_wd[g][r];
+    sh.step[g][r] = s_dev->step[g][r];
+    if (threadIdx.x == 0) {
+      sh.one_minus_beta1 = s_dev->one_minus_beta1; sh.one_minus_beta2 = s_dev->one_minus_beta2;
+      sh.rsqrt_bc2 = s_dev->rsqrt_bc2; sh.eps = s_dev->eps; sh.inv_n = s_dev->inv_n; sh.n_replicas = s_dev->n_replicas;
+    }
+  } else {
+    sh.lr_wd[g][r] = s_param.lr_wd[g][r];
+    sh.step[g][r] = s_param.step[g][r];
+    if (threadIdx.x == 0) {
+      sh.one_minus_beta1 = s_param.one_minus_beta1; sh.one_minus_beta2 = s_param.one_minus_beta2;
+      sh.rsqrt_bc2 = s_param.rsqrt_bc2; sh.eps = s_param.eps; sh.inv_n = s_param.inv_n; sh.n_replicas = s_param.n_replicas;
+    }
+  }
+  __syncthreads();
+}
+
 template <typename GradT, bool kAdam, bool kConv, bool kMean>
 __global__ void __launch_bounds__(kThreads, 2)
-fanout_kernel(const __grid_constant__ LaunchPlan plan, const __grid_constant__ StepScalars s) {
+fanout_kernel(const __grid_constant__ LaunchPlan plan, const __grid_constant__ StepScalars s_param) {
+  __shared__ StepScalars s;
+  stage_scalars(s, s_param, plan.scal_dev);
   const AdamConsts c{s.one_minus_beta1, s.one_minus_beta2, s.rsqrt_bc2, s.eps};
   bool bad = false;
   for (int t = blockIdx.x; t < plan.n_tiles; t += gridDim.x) {
@@ -421,7 +448,9 @@ __device__ __forceinline__ void tile_vector_shared(const TensorDesc& td, long lo
 
 template <typename GradT, bool kConv, bool kMean>
 __global__ void __launch_bounds__(kThreads, 3)
-fanout_shared_kernel(const __grid_constant__ LaunchPlan plan, const __grid_constant__ StepScalars s) {
+fanout_shared_kernel(const __grid_constant__ LaunchPlan plan, const __grid_constant__ StepScalars s_param) {
+  __shared__ StepScalars s;
+  stage_scalars(s, s_param, plan.scal_dev);
   const AdamConsts c{s.one_minus_beta1, s.one_minus_beta2, s.rsqrt_bc2, s.eps};
   bool bad = false;
   for (int t = blockIdx.x; t < plan.n_tiles; t += gridDim.x) {

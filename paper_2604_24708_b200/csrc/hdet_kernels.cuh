@@ -50,6 +50,7 @@ struct LaunchPlan {
   int n_tiles;
   int grid;            // CTAs to launch; each takes tiles blockIdx.x, blockIdx.x + grid, ...
   unsigned* status;    // device status word; bit 0 = non-finite parameter seen
+  const StepScalars* scal_dev;  // device-resident launch scalars; NULL = use the by-value kernel parameter
 };
 
 // Fan-out update of every replica of every tile (Eq. 2 or Adam); with `converge` the

@@ -25,7 +25,8 @@ class GpuRun:
     """The workload resident on the GPU, stepped through the C ABI."""
 
     def __init__(self, w: W.Workload, fuse: int = 1, shared_grad: bool = False, device: int = 0,
-                 grad_mean: bool = False, shared_state: bool = False):
+                 grad_mean: bool = False, shared_state: bool = False, device_resident: bool = False,
+                 loss_dtype: str = "float64"):
         import torch
         from hdet_inputs import device as D
         from paper_2604_24708_b200 import binding as B
@@ -42,6 +43,8 @@ class GpuRun:
         self.h = B.hdet_create(lib_config(B, w, fuse, device, 1 if grad_mean else 0), self.arena.descriptors())
         B.hdet_set_schedule(self.h, lib_schedule(B, w))
         self.i = 0
+        self.device_resident = device_resident
+        self.loss_buf = torch.zeros(w.n_replicas, dtype=getattr(torch, loss_dtype), device=f"cuda:{device}")
 
     def fill_grads(self, step: int) -> None:
         a, w = self.arena, self.w
@@ -59,9 +62,14 @@ class GpuRun:
         """One update with regenerated gradients and recipe losses; runs the controller after a sync."""
         self.fill_grads(self.i)
         losses = R.step_losses(self.w, self.i, perm0)
-        ended = self.B.hdet_step(self.h, list(losses))
-        if ended:
-            self.B.hdet_autolr_update(self.h)
+        if self.device_resident:
+            # the losses stay on the device; the controller runs there too
+            self.loss_buf.copy_(self.torch.from_numpy(np.asarray(losses)).to(self.loss_buf.dtype))
+            ended = self.B.hdet_step_device(self.h, self.loss_buf, self.torch.cuda.current_stream().cuda_stream)
+        else:
+            ended = self.B.hdet_step(self.h, list(losses))
+            if ended:
+                self.B.hdet_autolr_update(self.h)
         self.i += 1
         return ended
 
@@ -103,8 +111,10 @@ def oracle_for(w: W.Workload, params: Sequence[np.ndarray], groups: Sequence[int
 class OracleRun:
     """The oracle over chosen element ranges (slabs) of the workload, with the same seeded inputs."""
 
-    def __init__(self, w: W.Workload, slabs: Sequence[Slab], shared_grad: bool = False, grad_mean: bool = False):
+    def __init__(self, w: W.Workload, slabs: Sequence[Slab], shared_grad: bool = False, grad_mean: bool = False,
+                 loss_dtype: str = "float64"):
         self.w, self.slabs, self.shared_grad = w, list(slabs), shared_grad
+        self.loss_dtype = loss_dtype
         offs = w.arena_offsets()
         self.starts = [offs[k] + s for (k, s, n) in self.slabs]
         params = [np.tile(R.param_slab(w, a, n).astype(np.float64), (w.n_replicas, 1))
@@ -124,6 +134,8 @@ class OracleRun:
 
     def step(self) -> bool:
         losses = R.step_losses(self.w, self.i, self.o.perm_lr[0])
+        if self.loss_dtype == "float32":           # what the library reads from an fp32 loss tensor, exactly
+            losses = losses.astype(np.float32).astype(np.float64)
         ended = self.o.step(self.grads(self.i), losses)
         self.i += 1
         return ended

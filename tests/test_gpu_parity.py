@@ -19,10 +19,12 @@ TOL_ONE_STEP = 1e-6
 TOL_FULL_RUN = 1e-5
 
 
-def _lockstep(w, slabs, steps=None, fuse=1, shared_grad=False, check_every=None, grad_mean=False, shared_state=False):
+def _lockstep(w, slabs, steps=None, fuse=1, shared_grad=False, check_every=None, grad_mean=False, shared_state=False,
+              device_resident=False, loss_dtype="float64"):
     """Runs both sides for `steps` updates; checks after the first update, at chosen steps and at the end."""
-    g = H.GpuRun(w, fuse=fuse, shared_grad=shared_grad, grad_mean=grad_mean, shared_state=shared_state)
-    o = H.OracleRun(w, slabs, shared_grad=shared_grad, grad_mean=grad_mean)
+    g = H.GpuRun(w, fuse=fuse, shared_grad=shared_grad, grad_mean=grad_mean, shared_state=shared_state,
+                 device_resident=device_resident, loss_dtype=loss_dtype)
+    o = H.OracleRun(w, slabs, shared_grad=shared_grad, grad_mean=grad_mean, loss_dtype=loss_dtype)
     steps = steps or w.total_steps
     worst = 0.0
     try:
@@ -89,8 +91,9 @@ def test_shared_gradient_stride_zero():
     _lockstep(w, H.whole_tensor_slabs(w), shared_grad=True, check_every=4)
 
 
-def _final_arena(w, fuse=1, shared_grad=False, steps=None, grad_mean=False, shared_state=False):
-    g = H.GpuRun(w, fuse=fuse, shared_grad=shared_grad, grad_mean=grad_mean, shared_state=shared_state)
+def _final_arena(w, fuse=1, shared_grad=False, steps=None, grad_mean=False, shared_state=False, device_resident=False):
+    g = H.GpuRun(w, fuse=fuse, shared_grad=shared_grad, grad_mean=grad_mean, shared_state=shared_state,
+                 device_resident=device_resident)
     for i in range(steps or w.total_steps):
         g.step(g.perm0())
     a = g.arena
@@ -150,6 +153,95 @@ def test_config2_shape_with_gradient_mean_and_shared_moments_sampled():
     slabs = [(k, 0, min(2048, t.numel)) for k, t in enumerate(w.tensors) if k % 4 < 2]
     slabs += [(0, 2097152 - 4096, 4096), (10, 1024 * 1024 + 2048 * 7, 2048)]
     _lockstep(w, slabs, check_every=100, grad_mean=True, shared_state=True)
+
+
+@pytest.mark.parametrize("optimizer,grad_dtype", [(W.OPT_ADAMW, W.DTYPE_BF16), (W.OPT_SGD, W.DTYPE_F32)])
+@pytest.mark.parametrize("loss_dtype", ["float64", "float32"])
+@pytest.mark.parametrize("fuse", [1, 0])
+def test_device_resident_stepping_every_element_and_every_scalar(optimizer, grad_dtype, loss_dtype, fuse):
+    """hdet_step_device: schedule, spread, loss accumulation and controller computed by device kernels."""
+    w = W.ragged_workload(n_replicas=5, optimizer=optimizer, grad_dtype=grad_dtype)
+    _lockstep(w, H.whole_tensor_slabs(w), check_every=1, device_resident=True, loss_dtype=loss_dtype, fuse=fuse)
+
+
+def test_device_resident_config2_shape_sampled_with_shared_moments():
+    w = replace(W.config2(), total_steps=200, warmup_steps=60, sync_interval=20)
+    slabs = [(k, 0, min(2048, t.numel)) for k, t in enumerate(w.tensors) if k % 6 < 2]
+    _lockstep(w, slabs, check_every=50, device_resident=True, grad_mean=True, shared_state=True)
+
+
+def test_device_resident_equals_host_stepping_and_mode_switches():
+    import torch
+    w = W.ragged_workload(n_replicas=4, numels=(4097, 2048, 33))
+    host, _ = _final_arena(w)
+    dev, _ = _final_arena(w, device_resident=True)
+    for a, b in zip(host, dev):
+        assert H.rel_err(b.cpu().numpy(), a.cpu().numpy().astype(np.float64)).max() <= 1e-6
+    # a handle in device mode refuses host stepping until hdet_set_state hands the state back
+    g = H.GpuRun(w, device_resident=True)
+    for i in range(5):
+        g.step(g.perm0())
+    with pytest.raises(g.B.HdetError) as e:
+        g.B.hdet_step(g.h, None)
+    assert e.value.status == g.B.HDET_ERR_STATE
+    with pytest.raises(g.B.HdetError) as e:
+        g.B.hdet_autolr_update(g.h)
+    assert e.value.status == g.B.HDET_ERR_STATE
+    st = g.state()
+    assert st.step == 5
+    g.B.hdet_set_state(g.h, st)
+    g.device_resident = False
+    for i in range(5, w.total_steps):
+        g.step(g.perm0())
+    final = [g.arena.param.clone(), g.arena.exp_avg.clone(), g.arena.exp_avg_sq.clone()]
+    g.close()
+    for a, b in zip(host, final):
+        assert H.rel_err(b.cpu().numpy(), a.cpu().numpy().astype(np.float64)).max() <= 1e-6
+
+
+def test_device_resident_round_replayed_from_a_cuda_graph():
+    """A round of T device-resident steps recorded once and replayed gives the same bits as direct calls."""
+    import torch
+    w = replace(W.ragged_workload(n_replicas=4, numels=(4097, 2048, 33)), total_steps=40, warmup_steps=8,
+                sync_interval=4)
+    T, rounds = w.sync_interval, 5
+    losses = torch.tensor([[3.0 - 0.05 * r + 0.01 * i for r in range(4)] for i in range(T)], dtype=torch.float64,
+                          device="cuda")
+
+    def direct():
+        g = H.GpuRun(w, device_resident=True)
+        g.fill_grads(0)
+        s = torch.cuda.current_stream().cuda_stream
+        for k in range(rounds * T):
+            g.B.hdet_step_device(g.h, losses[k % T], s)
+        torch.cuda.synchronize()
+        out = [g.arena.param.clone(), g.arena.exp_avg.clone(), g.arena.exp_avg_sq.clone()], g.state()
+        g.close()
+        return out
+
+    ref, ref_state = direct()
+    g = H.GpuRun(w, device_resident=True)
+    g.fill_grads(0)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        for k in range(T):                                   # first round directly (uploads the state)
+            g.B.hdet_step_device(g.h, losses[k], side.cuda_stream)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        for k in range(T):
+            g.B.hdet_step_device(g.h, losses[k], torch.cuda.current_stream().cuda_stream)
+    for _ in range(rounds - 1):
+        graph.replay()
+    torch.cuda.synchronize()
+    st = g.state()                                           # reads the device copy back; host knows the count again
+    assert st.step == rounds * T == ref_state.step
+    assert bytes(st) == bytes(ref_state)
+    for a, b in zip(ref, [g.arena.param, g.arena.exp_avg, g.arena.exp_avg_sq]):
+        assert torch.equal(a, b)
+    assert st.fired == 1
+    g.close()
 
 
 def test_alpha_zero_keeps_replicas_bitwise_identical():

@@ -146,6 +146,9 @@ def test_schedule_checks_and_call_order():
     with pytest.raises(B.HdetError):
         B.hdet_autolr_update(h)
     assert B.hdet_kernel_launches(h) == 0
+    with pytest.raises(B.HdetError) as e:              # device-resident stepping needs tensors on a device
+        B.hdet_step_device(h)
+    assert e.value.status == B.HDET_ERR_UNSUPPORTED
     B.hdet_converge(h)                                 # nothing to do without tensors
     B.hdet_destroy(h)
     B.hdet_destroy(None)
