@@ -349,3 +349,59 @@ class HdetOracle:
             for g in range(self.G):
                 self.perm_lr[g] = permutation(self.seed, k, 2 * g, self.n)               # Eq. 9
                 self.perm_wd[g] = permutation(self.seed, k, 2 * g + 1, self.n)
+
+
+# --------------------------------------------------------------------------- #
+# Section 3.5, Eq. 10: warm noisy initialisation
+# --------------------------------------------------------------------------- #
+WARM_STREAM = 0x5741524D  # ASCII "WARM": separates these draws from the permutation draws
+
+
+def warm_sigma(theta0: Sequence[np.ndarray], nu: float) -> float:
+    """Standard deviation of Eq. 10: nu * sqrt(||theta_bar_0||^2 / d), d = total number of parameters.
+
+    theta0 is the whole checkpoint as a list of tensors (the norm and d run over all of them).
+    """
+    norm2 = 0.0
+    d = 0
+    for t in theta0:
+        t = np.asarray(t, dtype=np.float64)
+        norm2 += float(np.sum(t * t))
+        d += t.size
+    return nu * math.sqrt(norm2 / d)
+
+
+def warm_noise(seed: int, replica: int, tensor: int, start: int, n: int) -> np.ndarray:
+    """Standard normal draws epsilon_r / sigma of Eq. 10 for elements start .. start+n-1 of one tensor.
+
+    The paper asks for independent Gaussian noise per replica and parameter; the generator is this
+    repository's written definition (counter-based, so any element can be drawn on its own):
+    key = mix64(mix64(mix64(mix64(seed) + WARM_STREAM) + replica) + tensor); the element pair
+    p = e // 2 takes u = mix64(key + p * 0x9E3779B97F4A7C15), u1 = ((u >> 41) + 0.5) / 2**23,
+    u2 = ((u >> 16) & 0xFFFFFF) / 2**24, and the Box-Muller transform gives
+    z_even = sqrt(-2 ln u1) cos(2 pi u2), z_odd = sqrt(-2 ln u1) sin(2 pi u2).
+    """
+    key = mix64(mix64(mix64(mix64(seed) + WARM_STREAM) + replica) + tensor)
+    out = np.empty(n, dtype=np.float64)
+    for j in range(n):
+        e = start + j
+        u = mix64(key + (e // 2) * 0x9E3779B97F4A7C15)
+        u1 = ((u >> 41) + 0.5) / 8388608.0
+        u2 = ((u >> 16) & 0xFFFFFF) / 16777216.0
+        radius = math.sqrt(-2.0 * math.log(u1))
+        out[j] = radius * (math.cos(2.0 * math.pi * u2) if e % 2 == 0 else math.sin(2.0 * math.pi * u2))
+    return out
+
+
+def warm_noisy_init(theta0_slab: np.ndarray, sigma: float, seed: int, n_replicas: int, tensor: int,
+                    start: int = 0) -> np.ndarray:
+    """theta_r <- theta_bar_0 + epsilon_r, epsilon_r ~ N(0, sigma^2) independently per replica  (Eq. 10).
+
+    theta0_slab holds elements start .. of tensor `tensor` of the checkpoint; sigma comes from
+    warm_sigma over the whole checkpoint.  Returns an [N, len] array.
+    """
+    t0 = np.asarray(theta0_slab, dtype=np.float64)
+    out = np.empty((n_replicas, t0.size), dtype=np.float64)
+    for r in range(n_replicas):
+        out[r] = t0 + sigma * warm_noise(seed, r, tensor, start, t0.size)
+    return out

@@ -77,6 +77,16 @@ MUTANTS = [
     ("base[g] = self.ctrl_base[g] ", "base[g] = base_lr(self.sched_kind, self.i, self.S, self.ctrl_base[g], self.pct_start, self.div_factor, self.final_div_factor) "),
     ("sgd_update(th[r], g_r, lr[g_id][r])", "sgd_update(th[r], g_r, base[g_id])"),
     ("gk = g_bar / n", "gk = g_bar"),
+    # Eq. 10
+    ("return nu * math.sqrt(norm2 / d)", "return nu * math.sqrt(norm2) / d"),
+    ("return nu * math.sqrt(norm2 / d)", "return nu * norm2 / d"),
+    ("radius = math.sqrt(-2.0 * math.log(u1))", "radius = math.sqrt(-math.log(u1))"),
+    ("u2 = ((u >> 16) & 0xFFFFFF) / 16777216.0", "u2 = ((u >> 41) & 0xFFFFFF) / 16777216.0"),
+    ("out[j] = radius * (math.cos(2.0 * math.pi * u2) if e % 2 == 0 else math.sin(2.0 * math.pi * u2))",
+     "out[j] = radius * math.cos(2.0 * math.pi * u2)"),
+    ("u = mix64(key + (e // 2) * 0x9E3779B97F4A7C15)", "u = mix64(key + j * 0x9E3779B97F4A7C15)"),
+    ("out[r] = t0 + sigma * warm_noise(seed, r, tensor, start, t0.size)", "out[r] = t0 + sigma * warm_noise(seed, 0, tensor, start, t0.size)"),
+    ("out[r] = t0 + sigma * warm_noise(seed, r, tensor, start, t0.size)", "out[r] = t0 * (1 + sigma * warm_noise(seed, r, tensor, start, t0.size))"),
     ("if self.grad_mean and gk.ndim == 2:", "if False:"),
     ("lr[g_id][r], wd[g_id][r],", "lr[g_id][r], self.weight_decay[g_id],"),
 ]

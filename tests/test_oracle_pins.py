@@ -540,3 +540,51 @@ def test_alg1_gradient_mean_equals_a_run_with_the_mean_given_as_shared_gradient(
             assert np.allclose(a.v[k], b.v[k], rtol=1e-12, atol=1e-30)
             # one gradient for everyone: the moments are the same on every replica
             assert np.all(a.m[k] == a.m[k][0]) and np.all(a.v[k] == a.v[k][0])
+
+
+# ----------------------------------------------------------------------------- Eq. 10
+def test_eq10_sigma_matches_the_stated_variance():
+    rng = np.random.default_rng(20)
+    ts = [rng.normal(scale=0.02, size=1000), rng.normal(scale=0.5, size=37)]
+    flat = np.concatenate(ts)
+    # nu^2 ||theta||^2 / d written with a library norm
+    assert O.warm_sigma(ts, 0.01) ** 2 == pytest.approx(0.01 ** 2 * np.linalg.norm(flat) ** 2 / flat.size, rel=1e-12)
+    assert O.warm_sigma(ts, 0.0) == 0.0
+    assert O.warm_sigma([np.ones(10)], 0.01) == pytest.approx(0.01, rel=1e-14)   # unit-RMS checkpoint: sigma = nu
+    assert O.warm_sigma(ts, 0.02) == pytest.approx(2 * O.warm_sigma(ts, 0.01), rel=1e-14)
+
+
+def test_eq10_noise_is_standard_normal_and_independent():
+    from scipy import stats
+    z = O.warm_noise(3, 1, 0, 0, 40000)
+    assert abs(z.mean()) < 4 / np.sqrt(z.size) and abs(z.std() - 1) < 0.02
+    assert stats.kstest(z, "norm").pvalue > 1e-3                      # library normal distribution
+    assert abs(stats.kurtosis(z)) < 0.1 and abs(stats.skew(z)) < 0.05
+    # even and odd elements (the two Box-Muller outputs) are uncorrelated, as are replicas and tensors
+    assert abs(np.corrcoef(z[0::2], z[1::2])[0, 1]) < 0.03
+    assert abs(np.corrcoef(z[:10000], O.warm_noise(3, 2, 0, 0, 10000))[0, 1]) < 0.04
+    assert abs(np.corrcoef(z[:10000], O.warm_noise(3, 1, 1, 0, 10000))[0, 1]) < 0.04
+    assert abs(np.corrcoef(z[:10000], O.warm_noise(4, 1, 0, 0, 10000))[0, 1]) < 0.04
+    # counter-based: a slab equals the same elements of a longer draw, also from an odd start
+    assert np.array_equal(O.warm_noise(3, 1, 0, 1001, 50), z[1001:1051])
+    # the pair shares its radius: z_even^2 + z_odd^2 = -2 ln u1 is chi-square with 2 degrees of freedom
+    r2 = z[0::2] ** 2 + z[1::2] ** 2
+    assert stats.kstest(r2, "chi2", args=(2,)).pvalue > 1e-3
+
+
+def test_eq10_warm_init_statistics_and_limits():
+    rng = np.random.default_rng(21)
+    theta0 = rng.normal(scale=0.02, size=20000)
+    sigma = O.warm_sigma([theta0], 0.01)
+    out = O.warm_noisy_init(theta0, sigma, 9, 4, 0)
+    assert out.shape == (4, 20000)
+    eps = out - theta0
+    assert eps.std() == pytest.approx(0.01 * np.sqrt(np.mean(theta0 ** 2)), rel=0.02)     # nu * RMS(theta_0)
+    assert abs(eps.mean()) < 4 * sigma / np.sqrt(eps.size)
+    assert not np.allclose(out[0], out[1])
+    assert np.array_equal(O.warm_noisy_init(theta0, 0.0, 9, 4, 0), np.tile(theta0, (4, 1)))   # nu = 0: plain copies
+    # linear in sigma
+    out2 = O.warm_noisy_init(theta0, 2 * sigma, 9, 4, 0)
+    assert np.allclose(out2 - theta0, 2 * eps, rtol=1e-9, atol=1e-16)
+    # a slab of the tensor gives the same values as the whole tensor
+    assert np.array_equal(O.warm_noisy_init(theta0[333:444], sigma, 9, 4, 0, start=333), out[:, 333:444])
