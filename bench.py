@@ -341,6 +341,11 @@ def run_ours(args):
             if label == "fanout_update":
                 ms = timed(lambda: B.hdet_converge(hk, stream.cuda_stream))
                 per_kernel["converge_standalone"] = {"ms": ms, "GB_per_s": 8 * n * P / ms / 1e6, "bytes_per_element": 8}
+            if label == "fanout_update":
+                # Eq. 10 (three kernels): reads the checkpoint twice (norm, then fan-out) and writes all N replicas
+                ms = timed(lambda: B.hdet_warm_init(hk, 0.01, 1, stream.cuda_stream), reps=3)
+                wb = (8 + 4 * n) * P
+                per_kernel["warm_init"] = {"ms": ms, "GB_per_s": wb / ms / 1e6, "bytes_per_element": wb / (n * P)}
             B.hdet_destroy(hk)
 
     if rank != 0:

@@ -219,6 +219,20 @@ HDET_API int hdet_step_device(hdet_handle h, const void* d_step_losses, int32_t 
                               int32_t* did_converge);
 
 /*
+ * hdet_warm_init -- warm noisy initialisation (Section 3.5, Eq. 10), to be called before the first
+ * update when training starts from a checkpoint.  Replica 0 of every tensor must hold the checkpoint
+ * theta_bar_0; on return (stream order) every replica r, replica 0 included, holds
+ * theta_bar_0 + eps_r with eps_r ~ N(0, nu^2 ||theta_bar_0||^2 / d), where the norm and d (the number
+ * of parameters) run over ALL tensors of the handle.  The noise is a counter-based Box-Muller draw
+ * keyed by (seed, replica, tensor index, element index), so it does not depend on layout or launch
+ * shape; nu = 0 copies the checkpoint to all replicas.  The paper uses nu = 0.01.
+ * Moments and the step count are not touched.  The first call allocates a scratch buffer of one
+ * double per 2048-element tile (freed by hdet_destroy); later calls allocate nothing.
+ * Errors: INVALID_ARG (nu negative or not finite), CUDA.
+ */
+HDET_API int hdet_warm_init(hdet_handle h, double nu, uint64_t seed, void* stream);
+
+/*
  * hdet_converge -- Eq. 3 on its own: theta_r <- (1/N) sum_r' theta_r' for every tensor.
  * Does not touch the step count, the moments or the loss accumulator.
  * Errors: INVALID_ARG, CUDA.

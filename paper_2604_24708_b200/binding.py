@@ -91,6 +91,8 @@ def _load() -> C.CDLL:
     lib.hdet_step.argtypes = [H, C.POINTER(C.c_double), C.c_void_p, C.POINTER(C.c_int32)]
     lib.hdet_step_device.argtypes = [H, C.c_void_p, C.c_int32, C.c_void_p, C.POINTER(C.c_int32)]
     lib.hdet_step_device.restype = C.c_int
+    lib.hdet_warm_init.argtypes = [H, C.c_double, C.c_uint64, C.c_void_p]
+    lib.hdet_warm_init.restype = C.c_int
     lib.hdet_converge.argtypes = [H, C.c_void_p]
     lib.hdet_autolr_update.argtypes = [H, C.POINTER(C.c_double), C.c_void_p]
     lib.hdet_get_state.argtypes = [H, C.POINTER(hdet_state)]
@@ -199,6 +201,11 @@ def hdet_step_device(h, d_step_losses=None, stream: int = 0) -> bool:
         ptr = C.c_void_p(d_step_losses.data_ptr())
     _check(_lib.hdet_step_device(h, ptr, dtype, C.c_void_p(stream), C.byref(flag)), h)
     return bool(flag.value)
+
+
+def hdet_warm_init(h, nu: float = 0.01, seed: int = 0, stream: int = 0) -> None:
+    """Eq. 10: every replica <- replica 0 (the checkpoint) + Gaussian noise of relative scale nu."""
+    _check(_lib.hdet_warm_init(h, nu, seed, C.c_void_p(stream)), h)
 
 
 def hdet_converge(h, stream: int = 0) -> None:

@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB_DIR = os.path.join(HERE, "lib")
 LIB_PATH = os.path.join(LIB_DIR, "libhdet.so")
-SOURCES = ["hdet_api.cu", "hdet_kernels.cu", "hdet_device_state.cu", "hdet_noalloc.cu"]
+SOURCES = ["hdet_api.cu", "hdet_kernels.cu", "hdet_device_state.cu", "hdet_noalloc.cu", "hdet_warm.cu"]
 HEADERS = ["hdet_kernels.cuh", "hdet_device_state.cuh", "hdet_scalars.h", "hdet_internal.h", os.path.join("..", "..", "include", "hdet.h")]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

@@ -44,6 +44,8 @@ struct hdet_ctx {
   TensorDesc* d_tensors = nullptr;
   Tile* d_tiles = nullptr;
   unsigned* d_status = nullptr;
+  double* d_warm = nullptr;      // scratch of hdet_warm_init (n_tiles + 1 doubles), allocated on its first call
+  double total_numel = 0.0;      // d of Eq. 10
   DevState* d_state = nullptr;   // device-resident scalar state (used by hdet_step_device)
   bool device_mode = false;      // the device copy of the state is the authoritative one
   int n_tiles = 0;
@@ -89,6 +91,8 @@ void free_device(hdet_ctx* h) {
   if (h->d_tiles) cudaFree(h->d_tiles);
   if (h->d_status) cudaFree(h->d_status);
   if (h->d_state) cudaFree(h->d_state);
+  if (h->d_warm) cudaFree(h->d_warm);
+  h->d_warm = nullptr;
   h->d_tensors = nullptr; h->d_tiles = nullptr; h->d_status = nullptr; h->d_state = nullptr;
 }
 
@@ -271,6 +275,7 @@ int hdet_create(const hdet_config* cfg, const hdet_tensor* tensors, int64_t n_te
   h->n_tensors = n_tensors;
   h->n_tiles = (int)tiles.size();
   h->shared_state = n_shared_state != 0;
+  for (int64_t k = 0; k < n_tensors; ++k) h->total_numel += (double)tensors[k].numel;
   spread_multipliers(n, cfg->alpha_lr, h->rho_lr);
   spread_multipliers(n, cfg->alpha_wd, h->rho_wd);
   for (int g = 0; g < HDET_MAX_GROUPS; ++g)
@@ -455,6 +460,24 @@ int hdet_step_device(hdet_handle h, const void* d_step_losses, int32_t loss_dtyp
   return HDET_OK;
 }
 
+int hdet_warm_init(hdet_handle h, double nu, uint64_t seed, void* stream) {
+  if (!h) return HDET_ERR_INVALID_ARG;
+  if (!(nu >= 0.0) || !std::isfinite(nu)) return fail(h, HDET_ERR_INVALID_ARG, "hdet_warm_init: nu must be finite and >= 0");
+  if (h->n_tiles == 0) return HDET_OK;
+  DeviceScope scope(h->cfg.device);
+  if (scope.err != cudaSuccess) return fail_cuda(h, "hdet_warm_init", scope.err);
+  if (!h->d_warm) {
+    cudaError_t e = cudaMalloc(&h->d_warm, sizeof(double) * ((size_t)h->n_tiles + 1));
+    if (e != cudaSuccess) return fail_cuda(h, "hdet_warm_init: scratch allocation", e);
+  }
+  LaunchPlan plan{h->d_tensors, h->d_tiles, h->n_tiles, h->grid_converge, h->d_status, nullptr};
+  cudaError_t e = launch_warm_init(plan, h->cfg.n_replicas, nu, h->total_numel, seed, h->d_warm,
+                                   static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return fail_cuda(h, "hdet_warm_init: launch", e);
+  h->launches += 3;
+  return HDET_OK;
+}
+
 int hdet_converge(hdet_handle h, void* stream) {
   if (!h) return HDET_ERR_INVALID_ARG;
   if (h->n_tiles == 0) return HDET_OK;
@@ -569,7 +592,7 @@ int hdet_set_state(hdet_handle h, const hdet_state* in) {
 
 int hdet_destroy(hdet_handle h) {
   if (!h) return HDET_OK;
-  if (h->d_tensors || h->d_tiles || h->d_status || h->d_state) {
+  if (h->d_tensors || h->d_tiles || h->d_status || h->d_state || h->d_warm) {
     DeviceScope scope(h->cfg.device);
     free_device(h);
   }

@@ -60,6 +60,11 @@ struct LaunchPlan {
 cudaError_t launch_fanout(int optimizer, int grad_dtype, bool converge, bool grad_mean, bool shared_state,
                           const LaunchPlan& plan, const StepScalars& s, cudaStream_t stream);
 
+// Eq. 10: every replica <- replica 0 + N(0, nu^2 ||replica 0||^2 / total_numel) noise.  `scratch` holds
+// n_tiles + 1 doubles.  Three launches.
+cudaError_t launch_warm_init(const LaunchPlan& plan, int n_replicas, double nu, double total_numel,
+                             unsigned long long seed, double* scratch, cudaStream_t stream);
+
 // Stand-alone Eq. 3.
 cudaError_t launch_converge(const LaunchPlan& plan, int n_replicas, cudaStream_t stream);
 

@@ -367,3 +367,68 @@ def test_config5_n16_weight_decay_spread(T):
     if _free_gb() < 32:
         pytest.skip("needs 32 GB of free device memory")
     _lockstep(w, _decoder_sample(w, 6, 5), check_every=100)
+
+
+@pytest.mark.parametrize("align", [8, 1])
+def test_warm_noisy_init_every_element(align):
+    """Eq. 10 on the device against the oracle's counter-based Box-Muller draws; nu = 0; determinism."""
+    import torch
+    from oracle import hdet_oracle as O
+    w = W.ragged_workload(n_replicas=4, align_elems=align, numels=(4099, 7, 2048, 1, 6150, 33))
+    g = H.GpuRun(w)
+    offs = g.arena.offsets
+    theta0 = [g.arena.param[0, o:o + t.numel].cpu().numpy().astype(np.float64) for o, t in zip(offs, w.tensors)]
+    m_before = g.arena.exp_avg.clone()
+    g.B.hdet_warm_init(g.h, 0.01, 77)
+    sigma = O.warm_sigma(theta0, 0.01)
+    worst = 0.0
+    for k, (o, t) in enumerate(zip(offs, w.tensors)):
+        ref = O.warm_noisy_init(theta0[k], sigma, 77, 4, k)
+        got = g.arena.param[:, o:o + t.numel].cpu().numpy()
+        worst = max(worst, H.rel_err(got, ref).max())
+        # the noise itself, not just theta + noise: compare eps / sigma with the oracle's draws
+        z_got = (got.astype(np.float64) - theta0[k]) / sigma
+        z_ref = (ref - theta0[k]) / sigma
+        assert np.max(np.abs(z_got - z_ref)) < 2e-3          # fp32 rounding of theta + eps limits what can be resolved
+    assert worst <= TOL_ONE_STEP
+    assert torch.equal(g.arena.exp_avg, m_before) and g.state().step == 0
+    first = g.arena.param.clone()
+    # same seed on the perturbed replica 0 differs; restore the checkpoint and repeat: bitwise identical
+    for k, (o, t) in enumerate(zip(offs, w.tensors)):
+        g.arena.param[0, o:o + t.numel] = torch.from_numpy(theta0[k]).float().cuda()
+    g.B.hdet_warm_init(g.h, 0.01, 77)
+    assert torch.equal(g.arena.param, first)
+    # nu = 0: every replica is an exact copy of the checkpoint
+    for k, (o, t) in enumerate(zip(offs, w.tensors)):
+        g.arena.param[0, o:o + t.numel] = torch.from_numpy(theta0[k]).float().cuda()
+    g.B.hdet_warm_init(g.h, 0.0, 77)
+    for k, (o, t) in enumerate(zip(offs, w.tensors)):
+        blk = g.arena.param[:, o:o + t.numel]
+        assert torch.equal(blk, blk[0:1].expand_as(blk))
+        assert np.array_equal(blk[0].cpu().numpy().astype(np.float64), theta0[k])
+    with pytest.raises(g.B.HdetError):
+        g.B.hdet_warm_init(g.h, -1.0, 0)
+    g.close()
+
+
+def test_warm_noisy_init_config2_statistics_and_sampled_parity():
+    from oracle import hdet_oracle as O
+    w = W.config2()
+    g = H.GpuRun(w)
+    n = w.n_replicas
+    offs = g.arena.offsets
+    theta0_full = g.arena.param[0].cpu().numpy().astype(np.float64)
+    theta0 = [theta0_full[o:o + t.numel] for o, t in zip(offs, w.tensors)]
+    g.B.hdet_warm_init(g.h, 0.01, 2024)
+    sigma = O.warm_sigma(theta0, 0.01)
+    assert sigma == pytest.approx(0.01 * 0.02, rel=2e-3)          # parameters are N(0, 0.02^2)
+    after = g.arena.param.cpu().numpy().astype(np.float64)
+    eps = after - theta0_full[None, :]
+    assert eps.std() == pytest.approx(sigma, rel=2e-3) and abs(eps.mean()) < 5 * sigma / np.sqrt(eps.size)
+    c = np.corrcoef(eps[0, :200000], eps[1, :200000])[0, 1]
+    assert abs(c) < 0.01                                           # replicas draw independent noise
+    for k, s0, ln in [(0, 0, 2048), (0, 2097152 - 3000, 3000), (1, 0, 2048), (22, 2048 * 500 + 1, 2047), (23, 5, 300)]:
+        ref = O.warm_noisy_init(theta0[k][s0:s0 + ln], sigma, 2024, n, k, start=s0)
+        got = after[:, offs[k] + s0:offs[k] + s0 + ln]
+        assert H.rel_err(got, ref).max() <= TOL_ONE_STEP
+    g.close()
