@@ -164,6 +164,17 @@ def sgd_update(theta: np.ndarray, g: np.ndarray, lr: float) -> None:
     theta -= lr * g
 
 
+def sgd_momentum_update(theta: np.ndarray, buf: np.ndarray, g: np.ndarray, lr: float, wd: float, mu: float) -> None:
+    """SGD with weight decay and a momentum buffer, in place (an extension: Eq. 2 has neither).
+
+    The usual definition (as in torch.optim.SGD without dampening or Nesterov): g' = g + wd * theta,
+    buf <- mu * buf + g' (buf starts at zero), theta <- theta - eta_r * buf.  With wd = mu = 0 this is Eq. 2.
+    """
+    g_eff = g + wd * theta
+    buf[...] = mu * buf + g_eff
+    theta -= lr * buf
+
+
 def adamw_update(theta: np.ndarray, m: np.ndarray, v: np.ndarray, g: np.ndarray, lr: float, wd: float,
                  beta1: float, beta2: float, eps: float, t: int) -> None:
     """One Adam step with decoupled weight decay, in place; t is the 1-based update number.
@@ -238,7 +249,7 @@ class HdetOracle:
                  ctrl_beta: float = 0.9, ctrl_sigma: float = 0.1, ctrl_lambda: float = 0.5,
                  f_div: float = 25.0, f_final: float = 1.0, reshuffle: bool = True, seed: int = 0,
                  beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8,
-                 n_replicas: Optional[int] = None, grad_mean: bool = False):
+                 n_replicas: Optional[int] = None, grad_mean: bool = False, momentum: float = 0.0):
         self.theta = [np.array(p, dtype=np.float64, copy=True) for p in params]
         self.n = self.theta[0].shape[0] if self.theta else int(n_replicas)
         self.m = [np.zeros_like(p) for p in self.theta]
@@ -259,6 +270,7 @@ class HdetOracle:
         self.reshuffle, self.seed = bool(reshuffle), seed
         self.beta1, self.beta2, self.eps = beta1, beta2, eps
         self.grad_mean = bool(grad_mean)
+        self.momentum = momentum
         # Algorithm 1, Init
         self.i = 0
         self.fired = False
@@ -314,8 +326,10 @@ class HdetOracle:
                 gk = g_bar / n
             for r in range(n):
                 g_r = gk if gk.ndim == 1 else gk[r]
-                if self.optimizer == SGD:
+                if self.optimizer == SGD and self.momentum == 0.0 and wd[g_id][r] == 0.0:
                     sgd_update(th[r], g_r, lr[g_id][r])                                   # Eq. 2
+                elif self.optimizer == SGD:
+                    sgd_momentum_update(th[r], self.m[k][r], g_r, lr[g_id][r], wd[g_id][r], self.momentum)
                 else:
                     adamw_update(th[r], self.m[k][r], self.v[k][r], g_r, lr[g_id][r], wd[g_id][r],
                                  self.beta1, self.beta2, self.eps, t)

@@ -77,6 +77,12 @@ MUTANTS = [
     ("base[g] = self.ctrl_base[g] ", "base[g] = base_lr(self.sched_kind, self.i, self.S, self.ctrl_base[g], self.pct_start, self.div_factor, self.final_div_factor) "),
     ("sgd_update(th[r], g_r, lr[g_id][r])", "sgd_update(th[r], g_r, base[g_id])"),
     ("gk = g_bar / n", "gk = g_bar"),
+    # SGD extension
+    ("g_eff = g + wd * theta", "g_eff = g - wd * theta"),
+    ("buf[...] = mu * buf + g_eff", "buf[...] = mu * buf + (1 - mu) * g_eff"),
+    ("theta -= lr * buf", "theta -= lr * g_eff"),
+    ("sgd_momentum_update(th[r], self.m[k][r], g_r, lr[g_id][r], wd[g_id][r], self.momentum)",
+     "sgd_momentum_update(th[r], self.m[k][0], g_r, lr[g_id][r], wd[g_id][r], self.momentum)"),
     # Eq. 10
     ("return nu * math.sqrt(norm2 / d)", "return nu * math.sqrt(norm2) / d"),
     ("return nu * math.sqrt(norm2 / d)", "return nu * norm2 / d"),
@@ -88,7 +94,8 @@ MUTANTS = [
     ("out[r] = t0 + sigma * warm_noise(seed, r, tensor, start, t0.size)", "out[r] = t0 + sigma * warm_noise(seed, 0, tensor, start, t0.size)"),
     ("out[r] = t0 + sigma * warm_noise(seed, r, tensor, start, t0.size)", "out[r] = t0 * (1 + sigma * warm_noise(seed, r, tensor, start, t0.size))"),
     ("if self.grad_mean and gk.ndim == 2:", "if False:"),
-    ("lr[g_id][r], wd[g_id][r],", "lr[g_id][r], self.weight_decay[g_id],"),
+    ("self.v[k][r], g_r, lr[g_id][r], wd[g_id][r],", "self.v[k][r], g_r, lr[g_id][r], self.weight_decay[g_id],"),
+    ("g_r, lr[g_id][r], wd[g_id][r], self.momentum)", "g_r, lr[g_id][r], self.weight_decay[g_id], self.momentum)"),
 ]
 
 

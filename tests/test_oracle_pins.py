@@ -588,3 +588,47 @@ def test_eq10_warm_init_statistics_and_limits():
     assert np.allclose(out2 - theta0, 2 * eps, rtol=1e-9, atol=1e-16)
     # a slab of the tensor gives the same values as the whole tensor
     assert np.array_equal(O.warm_noisy_init(theta0[333:444], sigma, 9, 4, 0, start=333), out[:, 333:444])
+
+
+def test_sgd_momentum_and_weight_decay_match_the_library():
+    rng = np.random.default_rng(30)
+    n = 101
+    th0 = rng.normal(scale=0.02, size=n)
+    for mu, wd in [(0.9, 0.0), (0.9, 0.05), (0.0, 0.1), (0.5, 0.01)]:
+        th, buf = th0.copy(), np.zeros(n)
+        p = torch.nn.Parameter(torch.tensor(th0))
+        opt = torch.optim.SGD([p], lr=0.1, momentum=mu, weight_decay=wd)
+        for t in range(1, 9):
+            g = rng.normal(scale=1e-2, size=n)
+            lr = 1e-2 * (1 + t % 3)
+            O.sgd_momentum_update(th, buf, g, lr, wd, mu)
+            opt.param_groups[0]["lr"] = lr
+            p.grad = torch.tensor(g)
+            opt.step()
+            assert np.allclose(th, p.detach().numpy(), rtol=1e-12, atol=1e-18)
+    # mu = wd = 0 is Eq. 2
+    a, b, buf = th0.copy(), th0.copy(), np.zeros(n)
+    g = rng.normal(size=n)
+    O.sgd_momentum_update(a, buf, g, 0.3, 0.0, 0.0)
+    O.sgd_update(b, g, 0.3)
+    assert np.array_equal(a, b)
+
+
+def test_alg1_sgd_momentum_per_replica_rates_match_library_runs():
+    rng = np.random.default_rng(31)
+    n, ne, steps = 3, 7, 5
+    o = _mk(n, [ne], [0], 1, optimizer=O.SGD, sync_interval=100, total_steps=50, alpha_lr=0.3, alpha_wd=0.5,
+            weight_decay=[0.05], momentum=0.9)
+    th0 = o.theta[0][0].copy()
+    grads = rng.normal(scale=1e-2, size=(steps, n, ne))
+    for i in range(steps):
+        o.step([grads[i]])
+    rho, rho_wd = O.spread_multipliers(n, 0.3), O.spread_multipliers(n, 0.5)
+    for r in range(n):
+        p = torch.nn.Parameter(torch.tensor(th0))
+        opt = torch.optim.SGD([p], lr=1.0, momentum=0.9, weight_decay=0.05 * rho_wd[r])
+        for i in range(steps):
+            opt.param_groups[0]["lr"] = O.onecycle_lr(i, 50, 3e-4) * rho[r]
+            p.grad = torch.tensor(grads[i][r])
+            opt.step()
+        assert np.allclose(o.theta[0][r], p.detach().numpy(), rtol=1e-12, atol=1e-18)
