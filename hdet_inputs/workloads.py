@@ -51,6 +51,7 @@ class Workload:
     beta1: float = 0.9
     beta2: float = 0.999
     eps: float = 1e-8
+    momentum: float = 0.0   # SGD momentum (0 = plain Eq. 2)
     weight_decay: Tuple[float, ...] = (0.0,)
     # base schedule
     sched_kind: int = SCHED_CONSTANT

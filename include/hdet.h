@@ -71,7 +71,8 @@ typedef struct hdet_ctx* hdet_handle;
 typedef struct {
   void* param;          /* fp32 [N] x numel, replica stride param_stride                  */
   void* grad;           /* fp32 or bf16 (hdet_config.grad_dtype), replica stride grad_stride */
-  void* exp_avg;        /* fp32 Adam first moment,  replica stride state_stride; NULL for SGD */
+  void* exp_avg;        /* fp32 Adam first moment (SGD with momentum: the momentum buffer),
+                           replica stride state_stride; NULL for plain SGD               */
   void* exp_avg_sq;     /* fp32 Adam second moment, replica stride state_stride; NULL for SGD */
   int64_t numel;        /* elements per replica, > 0                                      */
   int64_t param_stride; /* elements between replicas of param (>= numel when N > 1)       */
@@ -96,7 +97,9 @@ typedef struct {
   int32_t optimizer;     /* HDET_OPT_SGD (Eq. 2) or HDET_OPT_ADAMW (Section 4.1)          */
   int32_t grad_dtype;    /* HDET_DTYPE_F32 or HDET_DTYPE_BF16                             */
   double beta1, beta2, eps; /* Adam constants (ignored by SGD)                            */
-  double momentum;       /* SGD momentum; must be 0 (Eq. 2 has none)                      */
+  double momentum;       /* SGD momentum mu, 0 <= mu < 1.  0 is Eq. 2.  mu > 0 (an extension, Eq. 2
+                            has none): g' = g + wd theta, buf = mu buf + g', theta -= lr buf, with
+                            buf in exp_avg (one copy per replica, starting at 0)             */
   double alpha_lr;       /* spread ratio alpha of Eq. 1 for the learning rate, 0 <= a < 1 */
   double alpha_wd;       /* spread ratio for the weight decay (Remark 1), 0 <= a < 1; 0 = none */
   int64_t sync_interval; /* T of Section 3.3, >= 1                                        */
@@ -160,9 +163,9 @@ typedef struct {
  * tensors may be NULL only when n_tensors == 0.  On success *out receives the handle;
  * on failure *out is NULL and nothing is left allocated.
  * Errors: INVALID_ARG (NULL, N/G/T/alpha out of range, numel <= 0, group out of range,
- * stride < numel with N > 1, missing moments for AdamW, state_stride 0 without a common
- * gradient), ALIGN, UNSUPPORTED (momentum != 0; some but not all tensors with
- * state_stride 0), CUDA.
+ * stride < numel with N > 1, missing moments for AdamW or missing buffer for SGD momentum,
+ * momentum out of range or given with AdamW, state_stride 0 without a common gradient),
+ * ALIGN, UNSUPPORTED (some but not all tensors with state_stride 0), CUDA.
  */
 HDET_API int hdet_create(const hdet_config* cfg, const hdet_tensor* tensors, int64_t n_tensors, hdet_handle* out);
 
@@ -182,8 +185,8 @@ HDET_API int hdet_set_schedule(hdet_handle h, const hdet_schedule* sched);
  *   base_g   = controller's eta_bar_g once it has fired, else schedule_g(t - 1)
  *   lr[g][r] = base_g * rho_{pi_g(r)}                 (Eq. 1, Section 3.2, Eq. 9)
  *   wd[g][r] = wd_g * rho'_{pi'_g(r)}                 (Remark 1; rho' uses alpha_wd)
- *   every replica of every tensor is updated in one kernel (Eq. 2, or Adam with
- *   decoupled weight decay: theta *= 1 - lr*wd; m, v moving averages; theta -=
+ *   every replica of every tensor is updated in one kernel (Eq. 2 -- with a weight decay
+ *   the SGD gradient is g + wd*theta --, or Adam with decoupled weight decay: theta *= 1 - lr*wd; m, v moving averages; theta -=
  *   lr * (m/(1-beta1^t)) / (sqrt(v/(1-beta2^t)) + eps))
  *   step_losses (HOST, N doubles, or NULL) are added to the round's accumulator
  *   if t mod T == 0 the replicas are averaged (Eq. 3) -- inside the same kernel when

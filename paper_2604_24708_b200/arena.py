@@ -23,7 +23,7 @@ from . import binding as B
 class StackedArena:
     def __init__(self, numels: Sequence[int], groups: Sequence[int], n_replicas: int, optimizer: int,
                  grad_dtype: int, device: str = "cuda:0", align_elems: int = 8, shared_grad: bool = False,
-                 shared_state: bool = False):
+                 shared_state: bool = False, sgd_momentum: bool = False):
         if not torch.cuda.is_available():
             raise RuntimeError("StackedArena needs a CUDA device (there is no CPU path)")
         self.numels = [int(x) for x in numels]
@@ -44,7 +44,8 @@ class StackedArena:
         adam = optimizer == B.HDET_OPT_ADAMW
         self.shared_state = bool(shared_state) and adam
         sshape = (self.p_pad,) if self.shared_state else (self.n, self.p_pad)
-        self.exp_avg = torch.zeros(sshape, dtype=torch.float32, device=self.device) if adam else None
+        self.exp_avg = (torch.zeros(sshape, dtype=torch.float32, device=self.device)
+                        if (adam or sgd_momentum) else None)     # Adam first moment, or the SGD momentum buffer
         self.exp_avg_sq = torch.zeros(sshape, dtype=torch.float32, device=self.device) if adam else None
         self.shared_grad = bool(shared_grad)
         gshape = (self.p_pad,) if shared_grad else (self.n, self.p_pad)
@@ -59,6 +60,7 @@ class StackedArena:
             t.grad = self.grad.data_ptr() + gsz * off
             if self.exp_avg is not None:
                 t.exp_avg = self.exp_avg.data_ptr() + 4 * off
+            if self.exp_avg_sq is not None:
                 t.exp_avg_sq = self.exp_avg_sq.data_ptr() + 4 * off
             t.numel = ne
             t.param_stride = self.p_pad
@@ -69,5 +71,5 @@ class StackedArena:
         return out
 
     def resident_bytes(self) -> int:
-        ts = [self.param, self.grad] + ([self.exp_avg, self.exp_avg_sq] if self.exp_avg is not None else [])
+        ts = [t for t in (self.param, self.grad, self.exp_avg, self.exp_avg_sq) if t is not None]
         return sum(t.numel() * t.element_size() for t in ts)

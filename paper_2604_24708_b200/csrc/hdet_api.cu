@@ -173,7 +173,7 @@ DevConst device_constants(const hdet_ctx* h) {
   c.total_steps = h->sched.total_steps;
   c.warmup_steps = h->sched.warmup_steps;
   c.sync_interval = h->cfg.sync_interval;
-  c.beta1 = h->cfg.beta1; c.beta2 = h->cfg.beta2; c.eps = h->cfg.eps;
+  c.beta1 = h->cfg.beta1; c.beta2 = h->cfg.beta2; c.eps = h->cfg.eps; c.momentum = h->cfg.momentum;
   c.alpha_lr = h->cfg.alpha_lr; c.alpha_wd = h->cfg.alpha_wd;
   c.pct_start = h->sched.pct_start; c.div_factor = h->sched.div_factor; c.final_div_factor = h->sched.final_div_factor;
   c.ctrl_beta = h->sched.beta; c.sigma = h->sched.sigma; c.lambda = h->sched.lambda;
@@ -211,7 +211,10 @@ int hdet_create(const hdet_config* cfg, const hdet_tensor* tensors, int64_t n_te
     if (!(cfg->beta1 >= 0.0 && cfg->beta1 < 1.0) || !(cfg->beta2 >= 0.0 && cfg->beta2 < 1.0) || !(cfg->eps >= 0.0))
       return fail(nullptr, HDET_ERR_INVALID_ARG, "hdet_create: need 0 <= beta1, beta2 < 1 and eps >= 0");
   }
-  if (cfg->momentum != 0.0) return fail(nullptr, HDET_ERR_UNSUPPORTED, "hdet_create: SGD momentum is not implemented");
+  if (!(cfg->momentum >= 0.0 && cfg->momentum < 1.0))
+    return fail(nullptr, HDET_ERR_INVALID_ARG, "hdet_create: need 0 <= momentum < 1");
+  if (cfg->momentum != 0.0 && cfg->optimizer != HDET_OPT_SGD)
+    return fail(nullptr, HDET_ERR_INVALID_ARG, "hdet_create: momentum applies to HDET_OPT_SGD only");
   if (cfg->grad_mode != HDET_GRAD_AS_GIVEN && cfg->grad_mode != HDET_GRAD_REPLICA_MEAN)
     return fail(nullptr, HDET_ERR_INVALID_ARG, "hdet_create: unknown grad_mode");
 
@@ -221,6 +224,7 @@ int hdet_create(const hdet_config* cfg, const hdet_tensor* tensors, int64_t n_te
   std::vector<Tile> tiles;
   int64_t n_shared_state = 0;
   const bool adamw = cfg->optimizer == HDET_OPT_ADAMW;
+  const bool sgd_momentum = cfg->optimizer == HDET_OPT_SGD && cfg->momentum != 0.0;
   for (int64_t k = 0; k < n_tensors; ++k) {
     const hdet_tensor& t = tensors[k];
     char where[64];
@@ -228,6 +232,9 @@ int hdet_create(const hdet_config* cfg, const hdet_tensor* tensors, int64_t n_te
     if (!t.param || !t.grad) return fail(nullptr, HDET_ERR_INVALID_ARG, std::string(where) + "param or grad is NULL");
     if (cfg->optimizer == HDET_OPT_ADAMW && (!t.exp_avg || !t.exp_avg_sq))
       return fail(nullptr, HDET_ERR_INVALID_ARG, std::string(where) + "AdamW needs exp_avg and exp_avg_sq");
+    if (sgd_momentum && (!t.exp_avg || (n > 1 && t.state_stride < t.numel)))
+      return fail(nullptr, HDET_ERR_INVALID_ARG, std::string(where) +
+                  "SGD with momentum needs exp_avg (the momentum buffer) with one copy per replica");
     if (t.numel <= 0) return fail(nullptr, HDET_ERR_INVALID_ARG, std::string(where) + "numel must be > 0");
     if (t.group < 0 || t.group >= cfg->n_groups)
       return fail(nullptr, HDET_ERR_INVALID_ARG, std::string(where) + "group out of range");
@@ -261,6 +268,7 @@ int hdet_create(const hdet_config* cfg, const hdet_tensor* tensors, int64_t n_te
     bool vec = aligned(t.param, 16) && aligned(t.grad, 4 * gsz) && t.param_stride % 4 == 0 && t.grad_stride % 4 == 0;
     if (cfg->optimizer == HDET_OPT_ADAMW)
       vec = vec && aligned(t.exp_avg, 16) && aligned(t.exp_avg_sq, 16) && t.state_stride % 4 == 0;
+    if (sgd_momentum) vec = vec && aligned(t.exp_avg, 16) && t.state_stride % 4 == 0;
     d.vec = vec ? 1 : 0;
     descs.push_back(d);
     for (int64_t j = 0; j < n_tiles_t; ++j) tiles.push_back(Tile{(int)k, (int)j});
@@ -362,13 +370,14 @@ int hdet_step(hdet_handle h, const double* step_losses, void* stream, int32_t* d
     }
     for (int g = 0; g < G; ++g)
       for (int r = 0; r < n; ++r) {
-        s.lr_wd[g][r] = adam ? (float)(h->lr[g][r] * h->wd[g][r]) : 0.0f;
+        s.lr_wd[g][r] = (float)(adam ? h->lr[g][r] * h->wd[g][r] : h->wd[g][r]);
         s.step[g][r] = (float)(adam ? h->lr[g][r] / bc1 : h->lr[g][r]);
       }
     s.one_minus_beta1 = (float)(1.0 - h->cfg.beta1);
     s.one_minus_beta2 = (float)(1.0 - h->cfg.beta2);
     s.rsqrt_bc2 = (float)(1.0 / std::sqrt(bc2));
     s.eps = (float)h->cfg.eps;
+    s.momentum = adam ? 0.0f : (float)h->cfg.momentum;
     s.inv_n = 1.0 / (double)n;
     s.n_replicas = n;
 
@@ -377,7 +386,8 @@ int hdet_step(hdet_handle h, const double* step_losses, void* stream, int32_t* d
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const bool fuse = ends_round && h->cfg.fuse_converge;
     LaunchPlan plan{h->d_tensors, h->d_tiles, h->n_tiles, h->grid_fanout, h->d_status, nullptr};
-    cudaError_t e = launch_fanout(h->cfg.optimizer, h->cfg.grad_dtype, fuse, h->cfg.grad_mode == HDET_GRAD_REPLICA_MEAN,
+    cudaError_t e = launch_fanout(h->cfg.optimizer, h->cfg.optimizer == HDET_OPT_SGD && h->cfg.momentum != 0.0, h->cfg.grad_dtype, fuse,
+                                  h->cfg.grad_mode == HDET_GRAD_REPLICA_MEAN,
                                   h->shared_state, plan, s, st);
     if (e != cudaSuccess) return fail_cuda(h, "hdet_step: fan-out launch", e);
     ++h->launches;
@@ -435,7 +445,8 @@ int hdet_step_device(hdet_handle h, const void* d_step_losses, int32_t loss_dtyp
   const bool fuse = ends_round && h->cfg.fuse_converge;
   LaunchPlan plan{h->d_tensors, h->d_tiles, h->n_tiles, h->grid_fanout, h->d_status, &h->d_state->scal};
   const StepScalars unused{};
-  e = launch_fanout(h->cfg.optimizer, h->cfg.grad_dtype, fuse, h->cfg.grad_mode == HDET_GRAD_REPLICA_MEAN,
+  e = launch_fanout(h->cfg.optimizer, h->cfg.optimizer == HDET_OPT_SGD && h->cfg.momentum != 0.0, h->cfg.grad_dtype, fuse,
+                                  h->cfg.grad_mode == HDET_GRAD_REPLICA_MEAN,
                     h->shared_state, plan, unused, st);
   if (e != cudaSuccess) return fail_cuda(h, "hdet_step_device: fan-out launch", e);
   ++h->launches;

@@ -40,7 +40,7 @@ __global__ void __launch_bounds__(32) device_scalars_kernel(DevState* d, const D
       const double wd = c.weight_decay[g] * spread_multiplier(c.n, c.alpha_wd, st.perm_wd[g][lane]);
       st.lr[g][lane] = lr;
       st.wd[g][lane] = wd;
-      sc.lr_wd[g][lane] = c.adam ? (float)(lr * wd) : 0.0f;
+      sc.lr_wd[g][lane] = (float)(c.adam ? lr * wd : wd);
       sc.step[g][lane] = (float)(c.adam ? lr / bc1 : lr);
     }
     if (lane == 0) st.base[g] = b;
@@ -56,6 +56,7 @@ __global__ void __launch_bounds__(32) device_scalars_kernel(DevState* d, const D
     sc.one_minus_beta2 = (float)(1.0 - c.beta2);
     sc.rsqrt_bc2 = (float)(1.0 / sqrt(bc2));
     sc.eps = (float)c.eps;
+    sc.momentum = c.adam ? 0.0f : (float)c.momentum;
     sc.inv_n = 1.0 / (double)c.n;
     sc.n_replicas = c.n;
     st.n_acc += 1;

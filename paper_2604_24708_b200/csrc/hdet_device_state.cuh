@@ -11,7 +11,7 @@ namespace hdet {
 struct DevConst {
   int n, n_groups, adam, kind, autolr, reshuffle;
   long long total_steps, warmup_steps, sync_interval;
-  double beta1, beta2, eps, alpha_lr, alpha_wd;
+  double beta1, beta2, eps, momentum, alpha_lr, alpha_wd;
   double pct_start, div_factor, final_div_factor;
   double ctrl_beta, sigma, lambda, f_div, f_final;
   double max_lr[HDET_MAX_GROUPS], weight_decay[HDET_MAX_GROUPS];

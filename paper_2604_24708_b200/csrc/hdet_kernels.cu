@@ -15,8 +15,10 @@
 namespace hdet {
 namespace {
 
+constexpr int kOptSgd = 0, kOptAdamW = 1, kOptSgdMomentum = 2;
+
 struct AdamConsts {
-  float one_minus_beta1, one_minus_beta2, rsqrt_bc2, eps;
+  float one_minus_beta1, one_minus_beta2, rsqrt_bc2, eps, momentum;
 };
 
 // Adam with decoupled weight decay on one element (Section 4.1 names Adam; weight decay is a
@@ -34,8 +36,18 @@ __device__ __forceinline__ void adam_element(float& th, float& m, float& v, floa
   th = fmaf(-step, m / denom, fmaf(-lr_wd, th, th));
 }
 
-// Eq. 2: theta <- theta - eta_r * g
-__device__ __forceinline__ void sgd_element(float& th, float g, float step) { th = fmaf(-step, g, th); }
+// Eq. 2: theta <- theta - eta_r * g.  With a weight decay the gradient is first extended by wd * theta
+// (the coupled form of SGD; wd = 0 leaves g untouched bit for bit).
+__device__ __forceinline__ void sgd_element(float& th, float g, float wd, float step) {
+  th = fmaf(-step, fmaf(wd, th, g), th);
+}
+
+// SGD with a momentum buffer (not part of Eq. 2; the usual definition): g' = g + wd theta;
+// buf = mu buf + g'; theta <- theta - eta_r buf.
+__device__ __forceinline__ void sgd_momentum_element(float& th, float& buf, float g, float wd, float step, float mu) {
+  buf = fmaf(mu, buf, fmaf(wd, th, g));
+  th = fmaf(-step, buf, th);
+}
 
 __device__ __forceinline__ bool not_finite(float x) { return !(fabsf(x) <= 3.402823466e38f); }
 
@@ -59,9 +71,10 @@ __device__ __forceinline__ float load_scalar(const __nv_bfloat16* p) {
 }
 
 // ---- scalar path: elements [begin, end) of one tensor, any alignment -----------------------
-template <typename GradT, bool kAdam, bool kConv, bool kMean>
+template <typename GradT, int kOpt, bool kConv, bool kMean>
 __device__ void range_scalar(const TensorDesc& td, long long begin, long long end, const StepScalars& s,
                              const AdamConsts& c, bool& bad) {
+  constexpr bool kAdam = kOpt == kOptAdamW, kMom = kOpt == kOptSgdMomentum;
   const int n = s.n_replicas;
   const GradT* grad = static_cast<const GradT*>(td.grad);
   for (long long e = begin + threadIdx.x; e < end; e += kThreads) {
@@ -81,8 +94,12 @@ __device__ void range_scalar(const TensorDesc& td, long long begin, long long en
         adam_element(th, m, v, g, s.lr_wd[td.group][r], s.step[td.group][r], c);
         __stcs(td.exp_avg + r * td.state_stride + e, m);
         __stcs(td.exp_avg_sq + r * td.state_stride + e, v);
+      } else if (kMom) {
+        float buf = __ldcs(td.exp_avg + r * td.state_stride + e);
+        sgd_momentum_element(th, buf, g, s.lr_wd[td.group][r], s.step[td.group][r], c.momentum);
+        __stcs(td.exp_avg + r * td.state_stride + e, buf);
       } else {
-        sgd_element(th, g, s.step[td.group][r]);
+        sgd_element(th, g, s.lr_wd[td.group][r], s.step[td.group][r]);
       }
       bad |= not_finite(th);
       if (kConv) sum += (double)th;
@@ -125,23 +142,24 @@ __device__ __forceinline__ void mean_gradient(const GradT* Gp, long long gs, con
     for (int q = 0; q < 4; ++q) gbar[k][q] = (float)(acc[k][q] * inv_n);
 }
 
-template <typename GradT, bool kAdam>
+template <typename GradT, int kOpt>
 struct ReplicaRegs {
   float4 th[kTileVecs];
-  float4 m[kAdam ? kTileVecs : 1];
-  float4 v[kAdam ? kTileVecs : 1];
+  float4 m[kOpt != kOptSgd ? kTileVecs : 1];        // Adam first moment, or the SGD momentum buffer
+  float4 v[kOpt == kOptAdamW ? kTileVecs : 1];
   typename GradRaw<GradT>::type g[kTileVecs];
 };
 
 // Processes `nvec` float4 vectors starting at element `off` of the tensor.  kFull: nvec == kThreads*kTileVecs.
-template <typename GradT, bool kAdam, bool kConv, bool kMean, bool kFull>
+template <typename GradT, int kOpt, bool kConv, bool kMean, bool kFull>
 __device__ __forceinline__ void tile_vector(const TensorDesc& td, long long off, int nvec, const StepScalars& s,
                                             const AdamConsts& c, bool& bad) {
-  using Regs = ReplicaRegs<GradT, kAdam>;
+  constexpr bool kAdam = kOpt == kOptAdamW, kMom = kOpt == kOptSgdMomentum;
+  using Regs = ReplicaRegs<GradT, kOpt>;
   const int n = s.n_replicas;
   const int grp = td.group;
   float* const P = td.param + off;
-  float* const M = kAdam ? td.exp_avg + off : nullptr;
+  float* const M = (kAdam || kMom) ? td.exp_avg + off : nullptr;
   float* const V = kAdam ? td.exp_avg_sq + off : nullptr;
   const GradT* const Gp = static_cast<const GradT*>(td.grad) + off;
   const long long ps = td.param_stride, gs = td.grad_stride, ss = td.state_stride;
@@ -160,14 +178,13 @@ __device__ __forceinline__ void tile_vector(const TensorDesc& td, long long off,
     for (int k = 0; k < kTileVecs; ++k) {
       if (ok[k]) {
         b.th[k] = __ldcs(reinterpret_cast<const float4*>(P + r * ps + idx[k]));
-        if (kAdam) {
-          b.m[k] = __ldcs(reinterpret_cast<const float4*>(M + r * ss + idx[k]));
-          b.v[k] = __ldcs(reinterpret_cast<const float4*>(V + r * ss + idx[k]));
-        }
+        if (kAdam || kMom) b.m[k] = __ldcs(reinterpret_cast<const float4*>(M + r * ss + idx[k]));
+        if (kAdam) b.v[k] = __ldcs(reinterpret_cast<const float4*>(V + r * ss + idx[k]));
         if (!kMean) b.g[k] = load_raw(Gp + r * gs + idx[k]);
       } else {
         b.th[k] = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (kAdam) { b.m[k] = b.th[k]; b.v[k] = b.th[k]; }
+        if (kAdam || kMom) b.m[k] = b.th[k];
+        if (kAdam) b.v[k] = b.th[k];
         b.g[k] = typename GradRaw<GradT>::type{};
       }
     }
@@ -210,9 +227,14 @@ __device__ __forceinline__ void tile_vector(const TensorDesc& td, long long off,
           __stcs(reinterpret_cast<float4*>(M + r * ss + idx[k]), make_float4(m[0], m[1], m[2], m[3]));
           __stcs(reinterpret_cast<float4*>(V + r * ss + idx[k]), make_float4(v[0], v[1], v[2], v[3]));
         }
+      } else if (kMom) {
+        float buf[4] = {b.m[k].x, b.m[k].y, b.m[k].z, b.m[k].w};
+#pragma unroll
+        for (int q = 0; q < 4; ++q) sgd_momentum_element(th[q], buf[q], g[q], lr_wd, step, c.momentum);
+        if (ok[k]) __stcs(reinterpret_cast<float4*>(M + r * ss + idx[k]), make_float4(buf[0], buf[1], buf[2], buf[3]));
       } else {
 #pragma unroll
-        for (int q = 0; q < 4; ++q) sgd_element(th[q], g[q], step);
+        for (int q = 0; q < 4; ++q) sgd_element(th[q], g[q], lr_wd, step);
       }
 #pragma unroll
       for (int q = 0; q < 4; ++q) bad |= not_finite(th[q]);
@@ -260,6 +282,7 @@ __device__ __forceinline__ void stage_scalars(StepScalars& sh, const StepScalars
     if (threadIdx.x == 0) {
       sh.one_minus_beta1 = s_dev->one_minus_beta1; sh.one_minus_beta2 = s_dev->one_minus_beta2;
       sh.rsqrt_bc2 = s_dev->rsqrt_bc2; sh.eps = s_dev->eps; sh.inv_n = s_dev->inv_n; sh.n_replicas = s_dev->n_replicas;
+      sh.momentum = s_dev->momentum;
     }
   } else {
     sh.lr_wd[g][r] = s_param.lr_wd[g][r];
@@ -267,17 +290,18 @@ __device__ __forceinline__ void stage_scalars(StepScalars& sh, const StepScalars
     if (threadIdx.x == 0) {
       sh.one_minus_beta1 = s_param.one_minus_beta1; sh.one_minus_beta2 = s_param.one_minus_beta2;
       sh.rsqrt_bc2 = s_param.rsqrt_bc2; sh.eps = s_param.eps; sh.inv_n = s_param.inv_n; sh.n_replicas = s_param.n_replicas;
+      sh.momentum = s_param.momentum;
     }
   }
   __syncthreads();
 }
 
-template <typename GradT, bool kAdam, bool kConv, bool kMean>
+template <typename GradT, int kOpt, bool kConv, bool kMean>
 __global__ void __launch_bounds__(kThreads, 2)
 fanout_kernel(const __grid_constant__ LaunchPlan plan, const __grid_constant__ StepScalars s_param) {
   __shared__ StepScalars s;
   stage_scalars(s, s_param, plan.scal_dev);
-  const AdamConsts c{s.one_minus_beta1, s.one_minus_beta2, s.rsqrt_bc2, s.eps};
+  const AdamConsts c{s.one_minus_beta1, s.one_minus_beta2, s.rsqrt_bc2, s.eps, s.momentum};
   bool bad = false;
   for (int t = blockIdx.x; t < plan.n_tiles; t += gridDim.x) {
     const Tile tile = plan.tiles[t];
@@ -287,14 +311,14 @@ fanout_kernel(const __grid_constant__ LaunchPlan plan, const __grid_constant__ S
     const int len = rest < kTileElems ? (int)rest : kTileElems;
     if (td.vec) {
       if (len == kTileElems) {
-        tile_vector<GradT, kAdam, kConv, kMean, true>(td, off, kThreads * kTileVecs, s, c, bad);
+        tile_vector<GradT, kOpt, kConv, kMean, true>(td, off, kThreads * kTileVecs, s, c, bad);
       } else {
         const int nvec = len >> 2;
-        if (nvec) tile_vector<GradT, kAdam, kConv, kMean, false>(td, off, nvec, s, c, bad);
-        if (len & 3) range_scalar<GradT, kAdam, kConv, kMean>(td, off + 4ll * nvec, off + len, s, c, bad);
+        if (nvec) tile_vector<GradT, kOpt, kConv, kMean, false>(td, off, nvec, s, c, bad);
+        if (len & 3) range_scalar<GradT, kOpt, kConv, kMean>(td, off + 4ll * nvec, off + len, s, c, bad);
       }
     } else {
-      range_scalar<GradT, kAdam, kConv, kMean>(td, off, off + len, s, c, bad);
+      range_scalar<GradT, kOpt, kConv, kMean>(td, off, off + len, s, c, bad);
     }
   }
   if (bad) atomicOr(plan.status, 1u);
@@ -451,7 +475,7 @@ __global__ void __launch_bounds__(kThreads, 3)
 fanout_shared_kernel(const __grid_constant__ LaunchPlan plan, const __grid_constant__ StepScalars s_param) {
   __shared__ StepScalars s;
   stage_scalars(s, s_param, plan.scal_dev);
-  const AdamConsts c{s.one_minus_beta1, s.one_minus_beta2, s.rsqrt_bc2, s.eps};
+  const AdamConsts c{s.one_minus_beta1, s.one_minus_beta2, s.rsqrt_bc2, s.eps, s.momentum};
   bool bad = false;
   for (int t = blockIdx.x; t < plan.n_tiles; t += gridDim.x) {
     const Tile tile = plan.tiles[t];
@@ -505,9 +529,9 @@ converge_kernel(const __grid_constant__ LaunchPlan plan, int n, double inv_n) {
   }
 }
 
-template <typename GradT, bool kAdam, bool kConv, bool kMean>
+template <typename GradT, int kOpt, bool kConv, bool kMean>
 cudaError_t launch_one(const LaunchPlan& plan, const StepScalars& s, cudaStream_t stream) {
-  fanout_kernel<GradT, kAdam, kConv, kMean><<<plan.grid, kThreads, 0, stream>>>(plan, s);
+  fanout_kernel<GradT, kOpt, kConv, kMean><<<plan.grid, kThreads, 0, stream>>>(plan, s);
   return cudaGetLastError();
 }
 
@@ -518,29 +542,31 @@ cudaError_t launch_shared(const LaunchPlan& plan, const StepScalars& s, cudaStre
 }
 
 template <typename GradT, bool kConv, bool kMean>
-cudaError_t pick_state(bool adam, bool shared_state, const LaunchPlan& plan, const StepScalars& s, cudaStream_t st) {
-  if (adam && shared_state) return launch_shared<GradT, kConv, kMean>(plan, s, st);
-  return adam ? launch_one<GradT, true, kConv, kMean>(plan, s, st) : launch_one<GradT, false, kConv, kMean>(plan, s, st);
+cudaError_t pick_state(int opt, bool shared_state, const LaunchPlan& plan, const StepScalars& s, cudaStream_t st) {
+  if (opt == kOptAdamW && shared_state) return launch_shared<GradT, kConv, kMean>(plan, s, st);
+  if (opt == kOptAdamW) return launch_one<GradT, kOptAdamW, kConv, kMean>(plan, s, st);
+  if (opt == kOptSgdMomentum) return launch_one<GradT, kOptSgdMomentum, kConv, kMean>(plan, s, st);
+  return launch_one<GradT, kOptSgd, kConv, kMean>(plan, s, st);
 }
 
 template <typename GradT>
-cudaError_t pick_flags(bool adam, bool converge, bool mean, bool shared_state, const LaunchPlan& plan,
+cudaError_t pick_flags(int opt, bool converge, bool mean, bool shared_state, const LaunchPlan& plan,
                        const StepScalars& s, cudaStream_t st) {
-  if (converge) return mean ? pick_state<GradT, true, true>(adam, shared_state, plan, s, st)
-                            : pick_state<GradT, true, false>(adam, shared_state, plan, s, st);
-  return mean ? pick_state<GradT, false, true>(adam, shared_state, plan, s, st)
-              : pick_state<GradT, false, false>(adam, shared_state, plan, s, st);
+  if (converge) return mean ? pick_state<GradT, true, true>(opt, shared_state, plan, s, st)
+                            : pick_state<GradT, true, false>(opt, shared_state, plan, s, st);
+  return mean ? pick_state<GradT, false, true>(opt, shared_state, plan, s, st)
+              : pick_state<GradT, false, false>(opt, shared_state, plan, s, st);
 }
 
 }  // namespace
 
-cudaError_t launch_fanout(int optimizer, int grad_dtype, bool converge, bool grad_mean, bool shared_state,
-                          const LaunchPlan& plan, const StepScalars& s, cudaStream_t stream) {
+cudaError_t launch_fanout(int optimizer, bool sgd_momentum, int grad_dtype, bool converge, bool grad_mean,
+                          bool shared_state, const LaunchPlan& plan, const StepScalars& s, cudaStream_t stream) {
   if (plan.n_tiles == 0) return cudaSuccess;
-  const bool adam = optimizer == HDET_OPT_ADAMW;
+  const int opt = optimizer == HDET_OPT_ADAMW ? kOptAdamW : (sgd_momentum ? kOptSgdMomentum : kOptSgd);
   if (grad_dtype == HDET_DTYPE_BF16)
-    return pick_flags<__nv_bfloat16>(adam, converge, grad_mean, shared_state, plan, s, stream);
-  return pick_flags<float>(adam, converge, grad_mean, shared_state, plan, s, stream);
+    return pick_flags<__nv_bfloat16>(opt, converge, grad_mean, shared_state, plan, s, stream);
+  return pick_flags<float>(opt, converge, grad_mean, shared_state, plan, s, stream);
 }
 
 cudaError_t launch_converge(const LaunchPlan& plan, int n_replicas, cudaStream_t stream) {

@@ -35,11 +35,12 @@ struct Tile {
 
 // Per-launch scalars, passed by value as kernel parameters (no device table to update).
 struct StepScalars {
-  float lr_wd[HDET_MAX_GROUPS][HDET_MAX_REPLICAS];  // lr * wd (decoupled decay factor is 1 - lr_wd)
+  float lr_wd[HDET_MAX_GROUPS][HDET_MAX_REPLICAS];  // AdamW: lr * wd (decoupled decay factor is 1 - lr_wd); SGD: wd
   float step[HDET_MAX_GROUPS][HDET_MAX_REPLICAS];   // AdamW: lr / (1 - beta1^t); SGD: lr
   float one_minus_beta1, one_minus_beta2;
   float rsqrt_bc2;  // 1 / sqrt(1 - beta2^t)
   float eps;
+  float momentum;   // SGD momentum (0 = none)
   double inv_n;     // 1 / N
   int n_replicas;
 };
@@ -57,8 +58,9 @@ struct LaunchPlan {
 // replica mean (Eq. 3) is formed from the updated values and written to all replicas.
 // `grad_mean`: every replica steps with the replica mean of the gradients (Algorithm 1's gradient
 // all-reduce).  `shared_state`: AdamW with one pair of moments for all replicas (state_stride 0).
-cudaError_t launch_fanout(int optimizer, int grad_dtype, bool converge, bool grad_mean, bool shared_state,
-                          const LaunchPlan& plan, const StepScalars& s, cudaStream_t stream);
+// `sgd_momentum`: SGD keeps a momentum buffer in exp_avg.
+cudaError_t launch_fanout(int optimizer, bool sgd_momentum, int grad_dtype, bool converge, bool grad_mean,
+                          bool shared_state, const LaunchPlan& plan, const StepScalars& s, cudaStream_t stream);
 
 // Eq. 10: every replica <- replica 0 + N(0, nu^2 ||replica 0||^2 / total_numel) noise.  `scratch` holds
 // n_tiles + 1 doubles.  Three launches.

@@ -35,7 +35,8 @@ class GpuRun:
         self.B, self.D, self.torch, self.w = B, D, torch, w
         self.arena = StackedArena([t.numel for t in w.tensors], [t.group for t in w.tensors], w.n_replicas,
                                   w.optimizer, w.grad_dtype, device=f"cuda:{device}", align_elems=w.align_elems,
-                                  shared_grad=shared_grad, shared_state=shared_state)
+                                  shared_grad=shared_grad, shared_state=shared_state,
+                                  sgd_momentum=(w.optimizer == W.OPT_SGD and w.momentum != 0.0))
         assert self.arena.offsets == w.arena_offsets()
         D.fill(self.arena.param[0], R.param_key(w), 0, R.param_scale(w))
         for r in range(1, w.n_replicas):
@@ -105,7 +106,7 @@ def oracle_for(w: W.Workload, params: Sequence[np.ndarray], groups: Sequence[int
         sync_interval=w.sync_interval, autolr=bool(w.autolr), warmup_steps=w.warmup_steps, ctrl_beta=w.ctrl_beta,
         ctrl_sigma=w.ctrl_sigma, ctrl_lambda=w.ctrl_lambda, f_div=w.f_div, f_final=w.f_final,
         reshuffle=bool(w.reshuffle), seed=w.seed, beta1=w.beta1, beta2=w.beta2, eps=w.eps, n_replicas=w.n_replicas,
-        grad_mean=grad_mean)
+        grad_mean=grad_mean, momentum=w.momentum)
 
 
 class OracleRun:
@@ -180,6 +181,8 @@ def compare_slabs(g: GpuRun, o: OracleRun, tol: float, check_moments: bool = Tru
         pairs = [("param", o.o.theta[idx])]
         if adam and check_moments:
             pairs += [("m", o.o.m[idx]), ("v", o.o.v[idx])]
+        if g.w.optimizer == W.OPT_SGD and g.w.momentum != 0.0 and check_moments:
+            pairs += [("m", o.o.m[idx])]
         for name, ref in pairs:
             got = g.slab(name, k, s, n)
             if got.shape[0] == 1 and ref.shape[0] > 1:       # shared moments: every oracle replica must agree

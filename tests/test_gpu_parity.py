@@ -244,6 +244,17 @@ def test_device_resident_round_replayed_from_a_cuda_graph():
     g.close()
 
 
+@pytest.mark.parametrize("grad_dtype", [W.DTYPE_F32, W.DTYPE_BF16])
+@pytest.mark.parametrize("align", [8, 1])
+@pytest.mark.parametrize("momentum,fuse", [(0.9, 1), (0.9, 0), (0.0, 1)])
+def test_sgd_with_weight_decay_and_momentum_every_element(grad_dtype, align, momentum, fuse):
+    """SGD beyond Eq. 2: coupled weight decay (spread per replica) and a momentum buffer per replica."""
+    w = replace(W.ragged_workload(n_replicas=4, optimizer=W.OPT_SGD, grad_dtype=grad_dtype, align_elems=align),
+                momentum=momentum)
+    _lockstep(w, H.whole_tensor_slabs(w), check_every=1, fuse=fuse)
+    _lockstep(w, H.whole_tensor_slabs(w), check_every=4, fuse=fuse, device_resident=True, grad_mean=True)
+
+
 def test_alpha_zero_keeps_replicas_bitwise_identical():
     import torch
     w = replace(W.ragged_workload(n_replicas=6, numels=(4097, 33)), alpha_lr=0.0, alpha_wd=0.0, autolr=0)

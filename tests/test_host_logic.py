@@ -75,9 +75,12 @@ def test_create_rejects_bad_config(kw):
 
 
 def test_create_rejects_momentum_and_bad_tensors_without_touching_a_device():
-    with pytest.raises(B.HdetError) as e:
-        B.hdet_create(_cfg(momentum=0.9, optimizer=B.HDET_OPT_SGD), [])
-    assert e.value.status == B.HDET_ERR_UNSUPPORTED
+    for kw in (dict(momentum=0.9), dict(momentum=1.0, optimizer=B.HDET_OPT_SGD), dict(momentum=-0.1, optimizer=B.HDET_OPT_SGD)):
+        with pytest.raises(B.HdetError) as e:
+            B.hdet_create(_cfg(**kw), [])                  # momentum with AdamW, or out of range
+        assert e.value.status == B.HDET_ERR_INVALID_ARG
+    h = B.hdet_create(_cfg(momentum=0.9, optimizer=B.HDET_OPT_SGD), [])
+    B.hdet_destroy(h)
 
     def tens(**kw):
         t = B.hdet_tensor(param=0x1000, grad=0x2000, exp_avg=0x3000, exp_avg_sq=0x4000, numel=100, param_stride=128,
@@ -85,6 +88,9 @@ def test_create_rejects_momentum_and_bad_tensors_without_touching_a_device():
         for k, v in kw.items():
             setattr(t, k, v)
         return t
+    with pytest.raises(B.HdetError) as e:                  # SGD with momentum needs its buffer
+        B.hdet_create(_cfg(momentum=0.9, optimizer=B.HDET_OPT_SGD), [tens(exp_avg=None)])
+    assert e.value.status == B.HDET_ERR_INVALID_ARG
     cases = [(dict(param=None), B.HDET_ERR_INVALID_ARG), (dict(grad=None), B.HDET_ERR_INVALID_ARG),
              (dict(exp_avg=None), B.HDET_ERR_INVALID_ARG), (dict(numel=0), B.HDET_ERR_INVALID_ARG),
              (dict(group=1), B.HDET_ERR_INVALID_ARG), (dict(group=-1), B.HDET_ERR_INVALID_ARG),
