@@ -113,6 +113,10 @@ typedef struct {
                             kernel first averages the N per-replica gradients of a tile and
                             every replica steps with that mean -- the single-GPU form of the
                             gradient all-reduce in Algorithm 1's loop                      */
+  int32_t n_replicas_global; /* 0: this handle holds all replicas.  > 0: the replica axis is sharded
+                            over GPUs; this handle holds n_replicas of n_replicas_global replicas
+                            (Eq. 1, Eq. 9 and the controller run over n_replicas_global <= 32)    */
+  int32_t replica_offset;    /* global index of this handle's replica 0 (sharded handles only)     */
 } hdet_config;
 
 /* Base schedule and controller constants (Algorithm 1, Require).  Host arrays with
@@ -196,6 +200,32 @@ HDET_API int hdet_set_schedule(hdet_handle h, const hdet_schedule* sched);
  * Errors: INVALID_ARG, STATE (no schedule), CUDA (launch failure).
  */
 HDET_API int hdet_step(hdet_handle h, const double* step_losses, void* stream, int32_t* did_converge);
+
+/*
+ * Replica axis sharded over GPUs (the paper's own arrangement, one or more replicas per GPU).
+ * Every rank creates a handle with n_replicas = its local replicas, n_replicas_global = N and its
+ * replica_offset, and per step:
+ *   hdet_step_sharded(h, losses of ALL N replicas (host, all-gathered by the caller), d_partial, ...)
+ *     -- like hdet_step; on the last update of a round the kernel does not write a mean but the
+ *        fp32 sums over the local replicas into d_partial (DEVICE, hdet_partial_layout elements,
+ *        16-byte aligned, caller-owned), and sets *did_converge;
+ *   the caller all-reduces d_partial (sum) over the ranks -- the one exchange of Eq. 3, P floats
+ *   per round, e.g. ncclAllReduce / torch.distributed.all_reduce on the same stream;
+ *   hdet_apply_mean(h, d_partial, stream) -- every local replica <- sum / N  (Eq. 3);
+ *   hdet_autolr_update(h, ...) as usual (every rank computes the same scalars from the same losses).
+ * The library itself calls no collective, so it has no dependency on a communication library and
+ * remote data is only ever read from local memory.  With a sharded handle hdet_step, hdet_converge
+ * and hdet_step_device return HDET_ERR_STATE / HDET_ERR_UNSUPPORTED, and grad_mode REPLICA_MEAN is
+ * refused (all-reduce the gradients and pass a shared gradient instead).  hdet_step_sharded also works
+ * on an unsharded handle (then hdet_apply_mean completes the converge locally).
+ * hdet_partial_layout: offsets[k] = element offset of tensor k in the staging buffer (multiples of 4;
+ * offsets may be NULL), *total_numel = its length.
+ * Errors: INVALID_ARG, ALIGN, STATE, CUDA.
+ */
+HDET_API int hdet_step_sharded(hdet_handle h, const double* step_losses, void* d_partial, void* stream,
+                               int32_t* did_converge);
+HDET_API int hdet_apply_mean(hdet_handle h, const void* d_sum, void* stream);
+HDET_API int hdet_partial_layout(hdet_handle h, int64_t* offsets, int64_t n_offsets, int64_t* total_numel);
 
 /*
  * hdet_step_device -- hdet_step and, at the end of a round, hdet_autolr_update, with Algorithm 1's

@@ -50,6 +50,7 @@ class hdet_config(C.Structure):
         ("alpha_lr", C.c_double), ("alpha_wd", C.c_double), ("sync_interval", C.c_int64),
         ("reshuffle", C.c_int32), ("fuse_converge", C.c_int32), ("seed", C.c_uint64),
         ("device", C.c_int32), ("grad_mode", C.c_int32),
+        ("n_replicas_global", C.c_int32), ("replica_offset", C.c_int32),
     ]
 
 
@@ -91,6 +92,12 @@ def _load() -> C.CDLL:
     lib.hdet_step.argtypes = [H, C.POINTER(C.c_double), C.c_void_p, C.POINTER(C.c_int32)]
     lib.hdet_step_device.argtypes = [H, C.c_void_p, C.c_int32, C.c_void_p, C.POINTER(C.c_int32)]
     lib.hdet_step_device.restype = C.c_int
+    lib.hdet_step_sharded.argtypes = [H, C.POINTER(C.c_double), C.c_void_p, C.c_void_p, C.POINTER(C.c_int32)]
+    lib.hdet_step_sharded.restype = C.c_int
+    lib.hdet_apply_mean.argtypes = [H, C.c_void_p, C.c_void_p]
+    lib.hdet_apply_mean.restype = C.c_int
+    lib.hdet_partial_layout.argtypes = [H, C.POINTER(C.c_int64), C.c_int64, C.POINTER(C.c_int64)]
+    lib.hdet_partial_layout.restype = C.c_int
     lib.hdet_warm_init.argtypes = [H, C.c_double, C.c_uint64, C.c_void_p]
     lib.hdet_warm_init.restype = C.c_int
     lib.hdet_converge.argtypes = [H, C.c_void_p]
@@ -201,6 +208,26 @@ def hdet_step_device(h, d_step_losses=None, stream: int = 0) -> bool:
         ptr = C.c_void_p(d_step_losses.data_ptr())
     _check(_lib.hdet_step_device(h, ptr, dtype, C.c_void_p(stream), C.byref(flag)), h)
     return bool(flag.value)
+
+
+def hdet_step_sharded(h, step_losses, d_partial, stream: int = 0) -> bool:
+    """One update of a handle that holds a shard of the replica axis; ``d_partial`` is a CUDA float32 tensor."""
+    flag = C.c_int32(0)
+    ptr = C.c_void_p(d_partial.data_ptr()) if d_partial is not None else None
+    _check(_lib.hdet_step_sharded(h, _doubles(step_losses), ptr, C.c_void_p(stream), C.byref(flag)), h)
+    return bool(flag.value)
+
+
+def hdet_apply_mean(h, d_sum, stream: int = 0) -> None:
+    _check(_lib.hdet_apply_mean(h, C.c_void_p(d_sum.data_ptr()), C.c_void_p(stream)), h)
+
+
+def hdet_partial_layout(h, n_tensors: int):
+    """(offsets per tensor, total elements) of the partial-sum staging buffer."""
+    offs = (C.c_int64 * max(1, n_tensors))()
+    total = C.c_int64(0)
+    _check(_lib.hdet_partial_layout(h, offs if n_tensors else None, n_tensors, C.byref(total)), h)
+    return list(offs)[:n_tensors], int(total.value)
 
 
 def hdet_warm_init(h, nu: float = 0.01, seed: int = 0, stream: int = 0) -> None:

@@ -52,6 +52,10 @@ struct hdet_ctx {
   int grid_fanout = 0;
   int grid_converge = 0;
   bool shared_state = false;   // AdamW with one pair of moments for all replicas
+  int n_global = 0;            // N of Eq. 1 over all GPUs (= cfg.n_replicas unless the replica axis is sharded)
+  int r_offset = 0;            // global index of local replica 0
+  int64_t partial_numel = 0;   // elements of the partial-sum staging buffer
+  std::vector<int64_t> partial_offsets;  // per tensor, inside that buffer
   int64_t launches = 0;
   std::string error;
 };
@@ -98,7 +102,7 @@ void free_device(hdet_ctx* h) {
 
 // Rates and weight decays for the update at 0-based index h->step.
 void compute_tables(hdet_ctx* h) {
-  const int n = h->cfg.n_replicas, G = h->cfg.n_groups;
+  const int n = h->n_global, G = h->cfg.n_groups;
   for (int g = 0; g < G; ++g) {
     const double b = h->fired ? h->ctrl_base[g]
                               : base_rate(h->sched.kind, h->step, h->sched.total_steps, h->max_lr[g],
@@ -164,7 +168,7 @@ void import_state(hdet_ctx* h, const hdet_state* in) {
 
 DevConst device_constants(const hdet_ctx* h) {
   DevConst c{};
-  c.n = h->cfg.n_replicas;
+  c.n = h->n_global;
   c.n_groups = h->cfg.n_groups;
   c.adam = h->cfg.optimizer == HDET_OPT_ADAMW;
   c.kind = h->sched.kind;
@@ -219,10 +223,19 @@ int hdet_create(const hdet_config* cfg, const hdet_tensor* tensors, int64_t n_te
     return fail(nullptr, HDET_ERR_INVALID_ARG, "hdet_create: unknown grad_mode");
 
   const int n = cfg->n_replicas;
+  const bool sharded = cfg->n_replicas_global != 0;
+  const int n_global = sharded ? cfg->n_replicas_global : n;
+  if (sharded && (cfg->replica_offset < 0 || n_global > HDET_MAX_REPLICAS || cfg->replica_offset + n > n_global))
+    return fail(nullptr, HDET_ERR_INVALID_ARG,
+                "hdet_create: need 0 <= replica_offset and replica_offset + n_replicas <= n_replicas_global <= 32");
+  if (sharded && cfg->grad_mode == HDET_GRAD_REPLICA_MEAN)
+    return fail(nullptr, HDET_ERR_UNSUPPORTED,
+                "hdet_create: with a sharded replica axis the gradient mean spans GPUs; all-reduce it and pass a shared gradient");
   const size_t gsz = cfg->grad_dtype == HDET_DTYPE_BF16 ? 2 : 4;
   std::vector<TensorDesc> descs;
   std::vector<Tile> tiles;
   int64_t n_shared_state = 0;
+  int64_t partial_numel = 0;
   const bool adamw = cfg->optimizer == HDET_OPT_ADAMW;
   const bool sgd_momentum = cfg->optimizer == HDET_OPT_SGD && cfg->momentum != 0.0;
   for (int64_t k = 0; k < n_tensors; ++k) {
@@ -270,6 +283,9 @@ int hdet_create(const hdet_config* cfg, const hdet_tensor* tensors, int64_t n_te
       vec = vec && aligned(t.exp_avg, 16) && aligned(t.exp_avg_sq, 16) && t.state_stride % 4 == 0;
     if (sgd_momentum) vec = vec && aligned(t.exp_avg, 16) && t.state_stride % 4 == 0;
     d.vec = vec ? 1 : 0;
+    d.partial_off = partial_numel;
+    d.partial = nullptr;
+    partial_numel += (t.numel + 3) / 4 * 4;
     descs.push_back(d);
     for (int64_t j = 0; j < n_tiles_t; ++j) tiles.push_back(Tile{(int)k, (int)j});
   }
@@ -284,8 +300,12 @@ int hdet_create(const hdet_config* cfg, const hdet_tensor* tensors, int64_t n_te
   h->n_tiles = (int)tiles.size();
   h->shared_state = n_shared_state != 0;
   for (int64_t k = 0; k < n_tensors; ++k) h->total_numel += (double)tensors[k].numel;
-  spread_multipliers(n, cfg->alpha_lr, h->rho_lr);
-  spread_multipliers(n, cfg->alpha_wd, h->rho_wd);
+  h->n_global = n_global;
+  h->r_offset = sharded ? cfg->replica_offset : 0;
+  h->partial_numel = partial_numel;
+  for (const TensorDesc& d : descs) h->partial_offsets.push_back(d.partial_off);
+  spread_multipliers(n_global, cfg->alpha_lr, h->rho_lr);
+  spread_multipliers(n_global, cfg->alpha_wd, h->rho_wd);
   for (int g = 0; g < HDET_MAX_GROUPS; ++g)
     for (int r = 0; r < HDET_MAX_REPLICAS; ++r) h->perm_lr[g][r] = h->perm_wd[g][r] = r;
 
@@ -349,13 +369,18 @@ int hdet_set_schedule(hdet_handle h, const hdet_schedule* s) {
   return HDET_OK;
 }
 
-int hdet_step(hdet_handle h, const double* step_losses, void* stream, int32_t* did_converge) {
+// One loop body of Algorithm 1 with host scalars.  `partial` != NULL: a round's last update writes the
+// sums over the local replicas to `partial` instead of the mean (replica axis sharded over GPUs).
+static int step_impl(hdet_handle h, const double* step_losses, bool sharded_call, float* partial, void* stream,
+                     int32_t* did_converge) {
   if (!h) return HDET_ERR_INVALID_ARG;
   if (did_converge) *did_converge = 0;
   if (!h->has_schedule) return fail(h, HDET_ERR_STATE, "hdet_step: call hdet_set_schedule first");
   if (h->device_mode)
     return fail(h, HDET_ERR_STATE, "hdet_step: the handle steps on the device (hdet_step_device); hdet_set_state returns it to host stepping");
-  const int n = h->cfg.n_replicas, G = h->cfg.n_groups;
+  if (!sharded_call && h->n_global != h->cfg.n_replicas)
+    return fail(h, HDET_ERR_STATE, "hdet_step: this handle holds a shard of the replica axis; use hdet_step_sharded and hdet_apply_mean");
+  const int n = h->cfg.n_replicas, n_all = h->n_global, off = h->r_offset, G = h->cfg.n_groups;
   compute_tables(h);
   const int64_t t = h->step + 1;
   const bool ends_round = (t % h->cfg.sync_interval) == 0;
@@ -370,8 +395,9 @@ int hdet_step(hdet_handle h, const double* step_losses, void* stream, int32_t* d
     }
     for (int g = 0; g < G; ++g)
       for (int r = 0; r < n; ++r) {
-        s.lr_wd[g][r] = (float)(adam ? h->lr[g][r] * h->wd[g][r] : h->wd[g][r]);
-        s.step[g][r] = (float)(adam ? h->lr[g][r] / bc1 : h->lr[g][r]);
+        const double lr = h->lr[g][off + r], wd = h->wd[g][off + r];   // local replica r is global replica off + r
+        s.lr_wd[g][r] = (float)(adam ? lr * wd : wd);
+        s.step[g][r] = (float)(adam ? lr / bc1 : lr);
       }
     s.one_minus_beta1 = (float)(1.0 - h->cfg.beta1);
     s.one_minus_beta2 = (float)(1.0 - h->cfg.beta2);
@@ -384,8 +410,9 @@ int hdet_step(hdet_handle h, const double* step_losses, void* stream, int32_t* d
     DeviceScope scope(h->cfg.device);
     if (scope.err != cudaSuccess) return fail_cuda(h, "hdet_step", scope.err);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const bool fuse = ends_round && h->cfg.fuse_converge;
-    LaunchPlan plan{h->d_tensors, h->d_tiles, h->n_tiles, h->grid_fanout, h->d_status, nullptr};
+    const bool fuse = ends_round && (h->cfg.fuse_converge || partial);
+    LaunchPlan plan{h->d_tensors, h->d_tiles, h->n_tiles, h->grid_fanout, h->d_status, nullptr,
+                    ends_round ? partial : nullptr};
     cudaError_t e = launch_fanout(h->cfg.optimizer, h->cfg.optimizer == HDET_OPT_SGD && h->cfg.momentum != 0.0, h->cfg.grad_dtype, fuse,
                                   h->cfg.grad_mode == HDET_GRAD_REPLICA_MEAN,
                                   h->shared_state, plan, s, st);
@@ -400,12 +427,12 @@ int hdet_step(hdet_handle h, const double* step_losses, void* stream, int32_t* d
   }
 
   if (step_losses)
-    for (int r = 0; r < n; ++r) h->loss_acc[r] += step_losses[r];
+    for (int r = 0; r < n_all; ++r) h->loss_acc[r] += step_losses[r];
   ++h->n_acc;
   h->step = t;
   h->round_ended = false;
   if (ends_round) {
-    for (int r = 0; r < n; ++r) {
+    for (int r = 0; r < n_all; ++r) {
       h->loss_round[r] = h->loss_acc[r] / (double)h->n_acc;
       h->loss_acc[r] = 0.0;
     }
@@ -416,10 +443,48 @@ int hdet_step(hdet_handle h, const double* step_losses, void* stream, int32_t* d
   return HDET_OK;
 }
 
+int hdet_step(hdet_handle h, const double* step_losses, void* stream, int32_t* did_converge) {
+  return step_impl(h, step_losses, false, nullptr, stream, did_converge);
+}
+
+int hdet_step_sharded(hdet_handle h, const double* step_losses, void* d_partial, void* stream, int32_t* did_converge) {
+  if (!h) return HDET_ERR_INVALID_ARG;
+  if (h->n_tiles > 0 && !d_partial) return fail(h, HDET_ERR_INVALID_ARG, "hdet_step_sharded: d_partial is NULL");
+  if (d_partial && !aligned(d_partial, 16))
+    return fail(h, HDET_ERR_ALIGN, "hdet_step_sharded: d_partial must be 16-byte aligned");
+  return step_impl(h, step_losses, true, static_cast<float*>(d_partial), stream, did_converge);
+}
+
+int hdet_apply_mean(hdet_handle h, const void* d_sum, void* stream) {
+  if (!h) return HDET_ERR_INVALID_ARG;
+  if (h->n_tiles == 0) return HDET_OK;
+  if (!d_sum || !aligned(d_sum, 16)) return fail(h, HDET_ERR_INVALID_ARG, "hdet_apply_mean: d_sum is NULL or not 16-byte aligned");
+  DeviceScope scope(h->cfg.device);
+  if (scope.err != cudaSuccess) return fail_cuda(h, "hdet_apply_mean", scope.err);
+  LaunchPlan plan{h->d_tensors, h->d_tiles, h->n_tiles, h->grid_converge, h->d_status, nullptr,
+                  const_cast<float*>(static_cast<const float*>(d_sum))};
+  cudaError_t e = launch_apply_mean(plan, h->cfg.n_replicas, 1.0 / (double)h->n_global, static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return fail_cuda(h, "hdet_apply_mean: launch", e);
+  ++h->launches;
+  return HDET_OK;
+}
+
+int hdet_partial_layout(hdet_handle h, int64_t* offsets, int64_t n_offsets, int64_t* total_numel) {
+  if (!h) return HDET_ERR_INVALID_ARG;
+  if (offsets && n_offsets != h->n_tensors)
+    return fail(h, HDET_ERR_INVALID_ARG, "hdet_partial_layout: n_offsets must equal the number of tensors");
+  if (offsets)
+    for (int64_t k = 0; k < h->n_tensors; ++k) offsets[k] = h->partial_offsets[k];
+  if (total_numel) *total_numel = h->partial_numel;
+  return HDET_OK;
+}
+
 int hdet_step_device(hdet_handle h, const void* d_step_losses, int32_t loss_dtype, void* stream, int32_t* did_converge) {
   if (!h) return HDET_ERR_INVALID_ARG;
   if (did_converge) *did_converge = 0;
   if (!h->has_schedule) return fail(h, HDET_ERR_STATE, "hdet_step_device: call hdet_set_schedule first");
+  if (h->n_global != h->cfg.n_replicas)
+    return fail(h, HDET_ERR_UNSUPPORTED, "hdet_step_device: not available when the replica axis is sharded over GPUs");
   if (h->n_tiles == 0 || !h->d_state)
     return fail(h, HDET_ERR_UNSUPPORTED, "hdet_step_device: the handle has no tensors, hence no device state");
   if (d_step_losses && loss_dtype != HDET_DTYPE_F32 && loss_dtype != HDET_DTYPE_F64)
@@ -482,7 +547,7 @@ int hdet_warm_init(hdet_handle h, double nu, uint64_t seed, void* stream) {
     if (e != cudaSuccess) return fail_cuda(h, "hdet_warm_init: scratch allocation", e);
   }
   LaunchPlan plan{h->d_tensors, h->d_tiles, h->n_tiles, h->grid_converge, h->d_status, nullptr};
-  cudaError_t e = launch_warm_init(plan, h->cfg.n_replicas, nu, h->total_numel, seed, h->d_warm,
+  cudaError_t e = launch_warm_init(plan, h->cfg.n_replicas, h->r_offset, nu, h->total_numel, seed, h->d_warm,
                                    static_cast<cudaStream_t>(stream));
   if (e != cudaSuccess) return fail_cuda(h, "hdet_warm_init: launch", e);
   h->launches += 3;
@@ -491,6 +556,8 @@ int hdet_warm_init(hdet_handle h, double nu, uint64_t seed, void* stream) {
 
 int hdet_converge(hdet_handle h, void* stream) {
   if (!h) return HDET_ERR_INVALID_ARG;
+  if (h->n_global != h->cfg.n_replicas)
+    return fail(h, HDET_ERR_UNSUPPORTED, "hdet_converge: this handle holds a shard of the replica axis; use hdet_step_sharded and hdet_apply_mean");
   if (h->n_tiles == 0) return HDET_OK;
   DeviceScope scope(h->cfg.device);
   if (scope.err != cudaSuccess) return fail_cuda(h, "hdet_converge", scope.err);
@@ -510,7 +577,7 @@ int hdet_autolr_update(hdet_handle h, const double* round_losses, void* /*stream
     return fail(h, HDET_ERR_STATE, "hdet_autolr_update: the last hdet_step did not end a round (or the update already ran)");
   h->round_ended = false;
   if (!h->sched.autolr || h->step < h->sched.warmup_steps) return HDET_OK;
-  const int n = h->cfg.n_replicas, G = h->cfg.n_groups;
+  const int n = h->n_global, G = h->cfg.n_groups;
   const double* L = round_losses ? round_losses : h->loss_round;
   for (int r = 0; r < n; ++r)
     if (!std::isfinite(L[r])) {
@@ -573,7 +640,7 @@ int hdet_set_state(hdet_handle h, const hdet_state* in) {
   if (!h) return HDET_ERR_INVALID_ARG;
   if (!in) return fail(h, HDET_ERR_INVALID_ARG, "hdet_set_state: in is NULL");
   if (in->step < 0 || in->n_acc < 0) return fail(h, HDET_ERR_INVALID_ARG, "hdet_set_state: negative step or n_acc");
-  const int n = h->cfg.n_replicas, G = h->cfg.n_groups;
+  const int n = h->n_global, G = h->cfg.n_groups;
   for (int g = 0; g < G; ++g)
     if (!is_permutation(in->perm_lr[g], n) || !is_permutation(in->perm_wd[g], n))
       return fail(h, HDET_ERR_INVALID_ARG, "hdet_set_state: a permutation array is not a permutation of 0..N-1");

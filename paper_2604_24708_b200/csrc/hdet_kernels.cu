@@ -106,8 +106,12 @@ __device__ void range_scalar(const TensorDesc& td, long long begin, long long en
       else __stcs(td.param + r * td.param_stride + e, th);
     }
     if (kConv) {
-      const float mean = (float)(sum * s.inv_n);
-      for (int r = 0; r < n; ++r) __stcs(td.param + r * td.param_stride + e, mean);
+      if (td.partial) {
+        td.partial[e] = (float)sum;       // replica axis sharded over GPUs: hand out the local sum instead
+      } else {
+        const float mean = (float)(sum * s.inv_n);
+        for (int r = 0; r < n; ++r) __stcs(td.param + r * td.param_stride + e, mean);
+      }
     }
   }
 }
@@ -262,6 +266,11 @@ __device__ __forceinline__ void tile_vector(const TensorDesc& td, long long off,
 #pragma unroll
     for (int k = 0; k < kTileVecs; ++k) {
       if (!ok[k]) continue;
+      if (td.partial) {   // replica axis sharded over GPUs: the local sum goes to the staging buffer
+        *reinterpret_cast<float4*>(td.partial + off + idx[k]) =
+            make_float4((float)sum[k][0], (float)sum[k][1], (float)sum[k][2], (float)sum[k][3]);
+        continue;
+      }
       const float4 mean = make_float4((float)(sum[k][0] * s.inv_n), (float)(sum[k][1] * s.inv_n),
                                       (float)(sum[k][2] * s.inv_n), (float)(sum[k][3] * s.inv_n));
       for (int rr = 0; rr < n; ++rr) __stcs(reinterpret_cast<float4*>(P + rr * ps + idx[k]), mean);
@@ -305,7 +314,8 @@ fanout_kernel(const __grid_constant__ LaunchPlan plan, const __grid_constant__ S
   bool bad = false;
   for (int t = blockIdx.x; t < plan.n_tiles; t += gridDim.x) {
     const Tile tile = plan.tiles[t];
-    const TensorDesc td = plan.tensors[tile.tensor];
+    TensorDesc td = plan.tensors[tile.tensor];
+    td.partial = plan.partial ? plan.partial + td.partial_off : nullptr;
     const long long off = (long long)tile.tile * kTileElems;
     const long long rest = td.numel - off;
     const int len = rest < kTileElems ? (int)rest : kTileElems;
@@ -363,8 +373,12 @@ __device__ void range_scalar_shared(const TensorDesc& td, long long begin, long 
       else __stcs(td.param + r * td.param_stride + e, th);
     }
     if (kConv) {
-      const float mean = (float)(sum * s.inv_n);
-      for (int r = 0; r < n; ++r) __stcs(td.param + r * td.param_stride + e, mean);
+      if (td.partial) {
+        td.partial[e] = (float)sum;       // replica axis sharded over GPUs: hand out the local sum instead
+      } else {
+        const float mean = (float)(sum * s.inv_n);
+        for (int r = 0; r < n; ++r) __stcs(td.param + r * td.param_stride + e, mean);
+      }
     }
   }
 }
@@ -463,9 +477,14 @@ __device__ __forceinline__ void tile_vector_shared(const TensorDesc& td, long lo
       }
     }
     if (kConv) {
-      const float4 mean = make_float4((float)(sum[0] * s.inv_n), (float)(sum[1] * s.inv_n),
-                                      (float)(sum[2] * s.inv_n), (float)(sum[3] * s.inv_n));
-      for (int rr = 0; rr < n; ++rr) __stcs(reinterpret_cast<float4*>(P + rr * ps + at), mean);
+      if (td.partial) {
+        *reinterpret_cast<float4*>(td.partial + off + at) =
+            make_float4((float)sum[0], (float)sum[1], (float)sum[2], (float)sum[3]);
+      } else {
+        const float4 mean = make_float4((float)(sum[0] * s.inv_n), (float)(sum[1] * s.inv_n),
+                                        (float)(sum[2] * s.inv_n), (float)(sum[3] * s.inv_n));
+        for (int rr = 0; rr < n; ++rr) __stcs(reinterpret_cast<float4*>(P + rr * ps + at), mean);
+      }
     }
   }
 }
@@ -479,7 +498,8 @@ fanout_shared_kernel(const __grid_constant__ LaunchPlan plan, const __grid_const
   bool bad = false;
   for (int t = blockIdx.x; t < plan.n_tiles; t += gridDim.x) {
     const Tile tile = plan.tiles[t];
-    const TensorDesc td = plan.tensors[tile.tensor];
+    TensorDesc td = plan.tensors[tile.tensor];
+    td.partial = plan.partial ? plan.partial + td.partial_off : nullptr;
     const long long off = (long long)tile.tile * kTileElems;
     const long long rest = td.numel - off;
     const int len = rest < kTileElems ? (int)rest : kTileElems;
@@ -529,6 +549,33 @@ converge_kernel(const __grid_constant__ LaunchPlan plan, int n, double inv_n) {
   }
 }
 
+// ---- second half of a converge whose replica axis is sharded over GPUs ----------------------------
+// plan.partial holds, per element, the sum over ALL replicas of all GPUs (the local sums after an
+// all-reduce); every local replica receives sum / N_global (Eq. 3).
+__global__ void __launch_bounds__(kThreads, 4)
+apply_mean_kernel(const __grid_constant__ LaunchPlan plan, int n_local, double inv_n_global) {
+  for (int t = blockIdx.x; t < plan.n_tiles; t += gridDim.x) {
+    const Tile tile = plan.tiles[t];
+    const TensorDesc td = plan.tensors[tile.tensor];
+    const long long off = (long long)tile.tile * kTileElems;
+    const long long rest = td.numel - off;
+    const int len = rest < kTileElems ? (int)rest : kTileElems;
+    const int nvec = td.vec ? (len >> 2) : 0;
+    float* const P = td.param + off;
+    const float* const S = plan.partial + td.partial_off + off;
+    for (int j = threadIdx.x; j < nvec; j += kThreads) {
+      const float4 x = __ldcs(reinterpret_cast<const float4*>(S + 4 * j));
+      const float4 mean = make_float4((float)(x.x * inv_n_global), (float)(x.y * inv_n_global),
+                                      (float)(x.z * inv_n_global), (float)(x.w * inv_n_global));
+      for (int r = 0; r < n_local; ++r) __stcs(reinterpret_cast<float4*>(P + r * td.param_stride + 4 * j), mean);
+    }
+    for (int e = 4 * nvec + threadIdx.x; e < len; e += kThreads) {
+      const float mean = (float)(__ldcs(S + e) * inv_n_global);
+      for (int r = 0; r < n_local; ++r) __stcs(P + r * td.param_stride + e, mean);
+    }
+  }
+}
+
 template <typename GradT, int kOpt, bool kConv, bool kMean>
 cudaError_t launch_one(const LaunchPlan& plan, const StepScalars& s, cudaStream_t stream) {
   fanout_kernel<GradT, kOpt, kConv, kMean><<<plan.grid, kThreads, 0, stream>>>(plan, s);
@@ -567,6 +614,12 @@ cudaError_t launch_fanout(int optimizer, bool sgd_momentum, int grad_dtype, bool
   if (grad_dtype == HDET_DTYPE_BF16)
     return pick_flags<__nv_bfloat16>(opt, converge, grad_mean, shared_state, plan, s, stream);
   return pick_flags<float>(opt, converge, grad_mean, shared_state, plan, s, stream);
+}
+
+cudaError_t launch_apply_mean(const LaunchPlan& plan, int n_local, double inv_n_global, cudaStream_t stream) {
+  if (plan.n_tiles == 0) return cudaSuccess;
+  apply_mean_kernel<<<plan.grid, kThreads, 0, stream>>>(plan, n_local, inv_n_global);
+  return cudaGetLastError();
 }
 
 cudaError_t launch_converge(const LaunchPlan& plan, int n_replicas, cudaStream_t stream) {

@@ -25,6 +25,8 @@ struct TensorDesc {
   long long state_stride;  // 0: one pair of moments shared by all replicas
   int group;
   int vec;  // 1: pointers and strides allow 128-bit accesses
+  long long partial_off;  // element offset of this tensor inside the partial-sum staging buffer (multiple of 4)
+  float* partial;         // set per tile by the kernels (NULL in the table)
 };
 
 // One unit of work: tile `tile` (kTileElems elements) of tensor `tensor`.
@@ -52,6 +54,7 @@ struct LaunchPlan {
   int grid;            // CTAs to launch; each takes tiles blockIdx.x, blockIdx.x + grid, ...
   unsigned* status;    // device status word; bit 0 = non-finite parameter seen
   const StepScalars* scal_dev;  // device-resident launch scalars; NULL = use the by-value kernel parameter
+  float* partial;      // non-NULL: a fused converge writes local replica sums here instead of the mean
 };
 
 // Fan-out update of every replica of every tile (Eq. 2 or Adam); with `converge` the
@@ -64,8 +67,11 @@ cudaError_t launch_fanout(int optimizer, bool sgd_momentum, int grad_dtype, bool
 
 // Eq. 10: every replica <- replica 0 + N(0, nu^2 ||replica 0||^2 / total_numel) noise.  `scratch` holds
 // n_tiles + 1 doubles.  Three launches.
-cudaError_t launch_warm_init(const LaunchPlan& plan, int n_replicas, double nu, double total_numel,
+cudaError_t launch_warm_init(const LaunchPlan& plan, int n_replicas, int replica_offset, double nu, double total_numel,
                              unsigned long long seed, double* scratch, cudaStream_t stream);
+
+// Every local replica <- plan.partial * inv_n_global (the all-reduced sums of a sharded converge).
+cudaError_t launch_apply_mean(const LaunchPlan& plan, int n_local, double inv_n_global, cudaStream_t stream);
 
 // Stand-alone Eq. 3.
 cudaError_t launch_converge(const LaunchPlan& plan, int n_replicas, cudaStream_t stream);

@@ -114,7 +114,7 @@ warm_noise_kernel(const __grid_constant__ LaunchPlan plan, const double* sigma_p
 
 }  // namespace
 
-cudaError_t launch_warm_init(const LaunchPlan& plan, int n_replicas, double nu, double total_numel,
+cudaError_t launch_warm_init(const LaunchPlan& plan, int n_replicas, int replica_offset, double nu, double total_numel,
                              unsigned long long seed, double* scratch, cudaStream_t stream) {
   if (plan.n_tiles == 0) return cudaSuccess;
   double* partial = scratch;                 // n_tiles partial sums
@@ -125,7 +125,8 @@ cudaError_t launch_warm_init(const LaunchPlan& plan, int n_replicas, double nu, 
   warm_sigma_kernel<<<1, 1024, 0, stream>>>(partial, plan.n_tiles, nu, total_numel, sigma);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  const unsigned long long base_key = mix64(mix64(seed) + 0x5741524Dull);
+  // local replica r draws the noise of global replica replica_offset + r
+  const unsigned long long base_key = mix64(mix64(seed) + 0x5741524Dull) + (unsigned long long)replica_offset;
   warm_noise_kernel<<<plan.grid, kThreads, 0, stream>>>(plan, sigma, n_replicas, base_key);
   return cudaGetLastError();
 }
