@@ -402,37 +402,63 @@ __device__ __forceinline__ void tile_vector_shared(const TensorDesc& td, long lo
     if (!kFull && j >= nvec) continue;
     const int at = j * 4;
 
-    // Parameters of up to kChunk replicas and both moments are requested first; the gradient (for the
-    // replica mean: N loads in groups of kGradChunk, summed in fp64) is consumed while they are in flight.
+    // All loads of the vector are requested before anything is consumed.  For the replica mean the N
+    // gradient loads come in groups of kG replicas whose fp64 sum needs the previous group, so the
+    // parameter loads are spread over the same groups: every wait covers a full wave of loads instead of
+    // a thin one of gradients only.
     float4 th[kChunk];
-#pragma unroll
-    for (int q = 0; q < kChunk; ++q)
-      th[q] = q < n ? __ldcs(reinterpret_cast<const float4*>(P + q * ps + at)) : make_float4(0.f, 0.f, 0.f, 0.f);
-    const float4 m4 = __ldcs(reinterpret_cast<const float4*>(M + at));
-    const float4 v4 = __ldcs(reinterpret_cast<const float4*>(V + at));
+    float4 m4, v4;
     float g[4];
     if constexpr (kMean) {
       double acc[4] = {0.0, 0.0, 0.0, 0.0};
       constexpr int kG = sizeof(typename GradRaw<GradT>::type) == 16 ? kGradChunk / 2 : kGradChunk;
-      for (int r0 = 0; r0 < n; r0 += kG) {
-        typename GradRaw<GradT>::type raw[kG];
+      m4 = __ldcs(reinterpret_cast<const float4*>(M + at));
+      v4 = __ldcs(reinterpret_cast<const float4*>(V + at));
 #pragma unroll
-        for (int q = 0; q < kG; ++q)
-          if (r0 + q < n) raw[q] = load_raw(Gp + (r0 + q) * gs + at);
+      for (int r0 = 0; r0 < kChunk; r0 += kG) {                      // replicas 0 .. kChunk-1, unrolled
+        typename GradRaw<GradT>::type raw[kG];
 #pragma unroll
         for (int q = 0; q < kG; ++q) {
           if (r0 + q < n) {
-            float gr[4];
-            unpack(raw[q], gr);
-#pragma unroll
-            for (int e = 0; e < 4; ++e) acc[e] += (double)gr[e];
+            raw[q] = load_raw(Gp + (r0 + q) * gs + at);
+            th[r0 + q] = __ldcs(reinterpret_cast<const float4*>(P + (r0 + q) * ps + at));
+          } else {
+            raw[q] = typename GradRaw<GradT>::type{};
+            th[r0 + q] = make_float4(0.f, 0.f, 0.f, 0.f);
           }
+        }
+        asm volatile("" ::: "memory");                                // keep the next group's loads after this wait
+#pragma unroll
+        for (int q = 0; q < kG; ++q) {
+          float gr[4];
+          unpack(raw[q], gr);
+#pragma unroll
+          for (int e = 0; e < 4; ++e) acc[e] += (double)gr[e];
+        }
+      }
+      for (int r0 = kChunk; r0 < n; r0 += kG) {                       // gradients of further replicas
+        typename GradRaw<GradT>::type raw[kG];
+#pragma unroll
+        for (int q = 0; q < kG; ++q)
+          raw[q] = r0 + q < n ? load_raw(Gp + (r0 + q) * gs + at) : typename GradRaw<GradT>::type{};
+#pragma unroll
+        for (int q = 0; q < kG; ++q) {
+          float gr[4];
+          unpack(raw[q], gr);
+#pragma unroll
+          for (int e = 0; e < 4; ++e) acc[e] += (double)gr[e];
         }
       }
 #pragma unroll
       for (int q = 0; q < 4; ++q) g[q] = (float)(acc[q] * s.inv_n);
+    } else {
+#pragma unroll
+      for (int q = 0; q < kChunk; ++q)
+        th[q] = q < n ? __ldcs(reinterpret_cast<const float4*>(P + q * ps + at)) : make_float4(0.f, 0.f, 0.f, 0.f);
+      m4 = __ldcs(reinterpret_cast<const float4*>(M + at));
+      v4 = __ldcs(reinterpret_cast<const float4*>(V + at));
+      unpack(load_raw(Gp + at), g);
     }
-    if constexpr (!kMean) unpack(load_raw(Gp + at), g);
 
     // Step direction u = m' / (sqrt(v')/sqrt(bc2) + eps), once per element for all replicas.
     float m[4] = {m4.x, m4.y, m4.z, m4.w};
