@@ -237,7 +237,8 @@ class HdetOracle:
       the weight decay (channel 2g + 1);
     * the losses are one per replica and shared by all groups;
     * weight decay is spread like the learning rate (Remark 1) with its own
-      ratio alpha_wd, but its base is not adapted by the controller;
+      ratio alpha_wd; its base is adapted by the same controller only with
+      auto_wd (Delta from the weight decays, same beta and lambda, gamma = 0);
     * eta_bar is not clamped.
     """
 
@@ -249,7 +250,8 @@ class HdetOracle:
                  ctrl_beta: float = 0.9, ctrl_sigma: float = 0.1, ctrl_lambda: float = 0.5,
                  f_div: float = 25.0, f_final: float = 1.0, reshuffle: bool = True, seed: int = 0,
                  beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8,
-                 n_replicas: Optional[int] = None, grad_mean: bool = False, momentum: float = 0.0):
+                 n_replicas: Optional[int] = None, grad_mean: bool = False, momentum: float = 0.0,
+                 auto_wd: bool = False):
         self.theta = [np.array(p, dtype=np.float64, copy=True) for p in params]
         self.n = self.theta[0].shape[0] if self.theta else int(n_replicas)
         self.m = [np.zeros_like(p) for p in self.theta]
@@ -286,6 +288,11 @@ class HdetOracle:
         self.base = None      # [G] base rates used by the last update
         self.w = None         # [N] softmax weights of the last controller firing
         self.delta = [0.0] * n_groups
+        # Remark 1: the same controller on the weight-decay channel (off unless auto_wd)
+        self.auto_wd = bool(auto_wd)
+        self.wd_base = list(weight_decay)      # h_bar of the weight-decay channel, per group
+        self.vel_wd = [0.0] * n_groups
+        self.delta_wd = [0.0] * n_groups
         self.L_round = None   # [N] mean losses of the last completed round
 
     def tables(self):
@@ -304,7 +311,7 @@ class HdetOracle:
                                   self.div_factor, self.final_div_factor)
             for r in range(n):
                 lr[g][r] = base[g] * rho[self.perm_lr[g][r]]             # Section 3.2; Eq. 9
-                wd[g][r] = self.weight_decay[g] * rho_wd[self.perm_wd[g][r]]
+                wd[g][r] = self.wd_base[g] * rho_wd[self.perm_wd[g][r]]
         return base, lr, wd
 
     def step(self, grads: Sequence[np.ndarray], losses: Optional[Sequence[float]] = None) -> bool:
@@ -357,6 +364,12 @@ class HdetOracle:
             tilde, bar, delta = hypergradient(self.w, self.lr[g])                        # Eq. 5, Eq. 6
             self.vel[g], self.ctrl_base[g] = meta_update(self.vel[g], bar, delta, self.beta, gamma, self.lam)  # Eq. 7
             self.delta[g] = delta
+            if self.auto_wd:
+                # Remark 1: Delta = h_tilde - h_bar with h the weight decays of the last update; the same
+                # velocity and gain; no decay term, since no floor is scheduled for the weight decay.
+                _, bar_wd, delta_wd = hypergradient(self.w, self.wd[g])
+                self.vel_wd[g], self.wd_base[g] = meta_update(self.vel_wd[g], bar_wd, delta_wd, self.beta, 0.0, self.lam)
+                self.delta_wd[g] = delta_wd
         self.fired = True
         if self.reshuffle:
             k = t // self.T

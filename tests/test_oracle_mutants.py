@@ -69,14 +69,19 @@ MUTANTS = [
     ("self.L_acc = np.zeros(n, dtype=np.float64)\n        self.n_acc = 0\n        if self.autolr", "if self.autolr"),
     ("self.L_round = self.L_acc / self.n_acc", "self.L_round = self.L_acc / self.T / 2"),
     ("lr[g][r] = base[g] * rho[self.perm_lr[g][r]]", "lr[g][r] = base[g] * rho[r]"),
-    ("wd[g][r] = self.weight_decay[g] * rho_wd[self.perm_wd[g][r]]", "wd[g][r] = self.weight_decay[g] * rho_wd[self.perm_lr[g][r]]"),
-    ("wd[g][r] = self.weight_decay[g] * rho_wd[self.perm_wd[g][r]]", "wd[g][r] = self.weight_decay[g] * rho[self.perm_wd[g][r]]"),
+    ("wd[g][r] = self.wd_base[g] * rho_wd[self.perm_wd[g][r]]", "wd[g][r] = self.wd_base[g] * rho_wd[self.perm_lr[g][r]]"),
+    ("wd[g][r] = self.wd_base[g] * rho_wd[self.perm_wd[g][r]]", "wd[g][r] = self.wd_base[g] * rho[self.perm_wd[g][r]]"),
     ("tilde, bar, delta = hypergradient(self.w, self.lr[g])", "tilde, bar, delta = hypergradient(self.w, self.lr[0])"),
     ("self.perm_wd[g] = permutation(self.seed, k, 2 * g + 1, self.n)", "self.perm_wd[g] = permutation(self.seed, k, 2 * g, self.n)"),
     ("        for th in self.theta:\n            converge(th)", "        for th in self.theta + self.m:\n            converge(th)"),
     ("base[g] = self.ctrl_base[g] ", "base[g] = base_lr(self.sched_kind, self.i, self.S, self.ctrl_base[g], self.pct_start, self.div_factor, self.final_div_factor) "),
     ("sgd_update(th[r], g_r, lr[g_id][r])", "sgd_update(th[r], g_r, base[g_id])"),
     ("gk = g_bar / n", "gk = g_bar"),
+    # Remark 1, weight-decay channel
+    ("_, bar_wd, delta_wd = hypergradient(self.w, self.wd[g])", "_, bar_wd, delta_wd = hypergradient(self.w, self.lr[g])"),
+    ("meta_update(self.vel_wd[g], bar_wd, delta_wd, self.beta, 0.0, self.lam)", "meta_update(self.vel_wd[g], bar_wd, delta_wd, self.beta, gamma, self.lam)"),
+    ("meta_update(self.vel_wd[g], bar_wd, delta_wd, self.beta, 0.0, self.lam)", "meta_update(self.vel[g], bar_wd, delta_wd, self.beta, 0.0, self.lam)"),
+    ("wd[g][r] = self.wd_base[g] * rho_wd[self.perm_wd[g][r]]", "wd[g][r] = self.weight_decay[g] * rho_wd[self.perm_wd[g][r]]"),
     # SGD extension
     ("g_eff = g + wd * theta", "g_eff = g - wd * theta"),
     ("buf[...] = mu * buf + g_eff", "buf[...] = mu * buf + (1 - mu) * g_eff"),

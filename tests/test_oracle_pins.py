@@ -632,3 +632,38 @@ def test_alg1_sgd_momentum_per_replica_rates_match_library_runs():
             p.grad = torch.tensor(grads[i][r])
             opt.step()
         assert np.allclose(o.theta[0][r], p.detach().numpy(), rtol=1e-12, atol=1e-18)
+
+
+def test_remark1_weight_decay_channel_controller():
+    n = 4
+    kw = dict(sync_interval=2, total_steps=40, autolr=True, warmup_steps=2, reshuffle=False, alpha_wd=0.5,
+              weight_decay=[0.05, 0.1], max_lr=[3e-4, 3e-4])
+    # identity permutation: replica r holds the r-th smallest weight decay; losses fall with r -> raise the base
+    up = _mk(n, [2, 2], [0, 1], 2, auto_wd=True, **kw)
+    down = _mk(n, [2, 2], [0, 1], 2, auto_wd=True, **kw)
+    flat = _mk(n, [2, 2], [0, 1], 2, auto_wd=True, **kw)
+    off = _mk(n, [2, 2], [0, 1], 2, auto_wd=False, **kw)
+    for i in range(8):
+        up.step([np.zeros(2)] * 2, 3.0 - 0.1 * np.linspace(-1, 1, n))
+        down.step([np.zeros(2)] * 2, 3.0 + 0.1 * np.linspace(-1, 1, n))
+        flat.step([np.zeros(2)] * 2, [3.0] * n)
+        off.step([np.zeros(2)] * 2, 3.0 - 0.1 * np.linspace(-1, 1, n))
+    assert up.wd_base[0] > 0.05 and down.wd_base[0] < 0.05 and up.delta_wd[0] > 0 > down.delta_wd[0]
+    assert flat.wd_base == pytest.approx([0.05, 0.1], rel=1e-14)              # equal losses: nothing moves (gamma = 0)
+    assert max(abs(v) for v in flat.vel_wd) < 1e-17
+    assert off.wd_base == [0.05, 0.1]
+    # linear in the weight decays: the group with twice the base gets twice Delta, velocity and base
+    assert up.delta_wd[1] == pytest.approx(2 * up.delta_wd[0], rel=1e-12)
+    assert up.wd_base[1] == pytest.approx(2 * up.wd_base[0], rel=1e-12)
+    # first firing by hand: two-replica-style closed form is covered by hypergradient; here Eq. 7 with gamma = 0
+    one = _mk(n, [2], [0], 1, auto_wd=True, sync_interval=2, total_steps=40, autolr=True, warmup_steps=2,
+              reshuffle=False, alpha_wd=0.5, weight_decay=[0.05])
+    L = 3.0 - 0.1 * np.linspace(-1, 1, n)
+    for i in range(2):
+        one.step([np.zeros(2)], L)
+    w = O.softmax_weights(L, 0.1)
+    delta = float(np.sum(w * 0.05 * O.spread_multipliers(n, 0.5))) - 0.05
+    assert one.wd_base[0] == pytest.approx(0.05 + 0.5 * 0.1 * delta, rel=1e-12)
+    # the tables of the next update use the new base
+    _, _, wd = one.tables()
+    assert wd[0].mean() == pytest.approx(one.wd_base[0], rel=1e-14)
