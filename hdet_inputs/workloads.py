@@ -73,6 +73,7 @@ class Workload:
     ctrl_lambda: float = 0.5
     f_div: float = 25.0
     f_final: float = 1.0
+    auto_wd: int = 0        # controller also on the weight-decay channel (Remark 1)
     # inputs
     seed: int = 1
     param_sigma: float = 0.02

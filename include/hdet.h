@@ -135,6 +135,10 @@ typedef struct {
   double sigma;            /* softmax temperature of Eq. 4, > 0                            */
   double lambda;           /* velocity gain of Eq. 7                                       */
   double f_div, f_final;   /* the two factors of Eq. 8, both > 0                           */
+  int32_t auto_wd;         /* 1 (with autolr): the controller also adapts each group's weight-decay
+                              base (Remark 1): Delta from the weight decays of the last update,
+                              the same beta and lambda, no decay term                       */
+  int32_t reserved;        /* set to 0                                                     */
 } hdet_schedule;
 
 /* Scalar state for logging and resume.  Tables are [group][replica]. */
@@ -158,6 +162,9 @@ typedef struct {
   double loss_acc[HDET_MAX_REPLICAS];  /* running sum of losses in the current round       */
   double loss_round[HDET_MAX_REPLICAS];/* mean loss per replica over the last full round   */
   double gamma;                        /* decay of Eq. 8                                   */
+  double wd_base[HDET_MAX_GROUPS];     /* base weight decay per group (adapted with auto_wd)   */
+  double wd_velocity[HDET_MAX_GROUPS]; /* velocity of the weight-decay channel (Remark 1)      */
+  double wd_delta[HDET_MAX_GROUPS];    /* its Delta at the last firing                         */
 } hdet_state;
 
 /*
@@ -177,7 +184,8 @@ HDET_API int hdet_create(const hdet_config* cfg, const hdet_tensor* tensors, int
  * hdet_set_schedule -- stores the base schedule eta(t) named in Algorithm 1's Require
  * list (one-cycle policy with cosine or linear annealing, or a constant) and the
  * controller constants (beta, sigma, lambda of Eq. 4 / Eq. 7; f_div, f_final of Eq. 8;
- * S_warm).  May be called again at any time; it does not reset the step count.
+ * S_warm).  May be called again at any time; it does not reset the step count, but it
+ * resets the base weight decays to sched->weight_decay.
  * Updates past step S keep the rate of step S - 1.
  * Errors: INVALID_ARG (NULL, S < 1, max_lr NULL, p*S <= 1 or p >= 1 for a one-cycle
  * kind, factors <= 0, sigma <= 0 with autolr, f_div or f_final <= 0).

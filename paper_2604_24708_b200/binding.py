@@ -60,7 +60,7 @@ class hdet_schedule(C.Structure):
         ("max_lr", C.POINTER(C.c_double)), ("weight_decay", C.POINTER(C.c_double)),
         ("pct_start", C.c_double), ("div_factor", C.c_double), ("final_div_factor", C.c_double),
         ("warmup_steps", C.c_int64), ("beta", C.c_double), ("sigma", C.c_double), ("lambda_", C.c_double),
-        ("f_div", C.c_double), ("f_final", C.c_double),
+        ("f_div", C.c_double), ("f_final", C.c_double), ("auto_wd", C.c_int32), ("reserved", C.c_int32),
     ]
 
 
@@ -77,6 +77,7 @@ class hdet_state(C.Structure):
         ("base", _GD), ("ctrl_base", _GD), ("velocity", _GD), ("delta", _GD),
         ("lr", _GND), ("wd", _GND), ("perm_lr", _GNI), ("perm_wd", _GNI),
         ("weights", _ND), ("loss_acc", _ND), ("loss_round", _ND), ("gamma", C.c_double),
+        ("wd_base", _GD), ("wd_velocity", _GD), ("wd_delta", _GD),
     ]
 
 
@@ -164,7 +165,7 @@ def tensor_from_torch(param, grad, exp_avg=None, exp_avg_sq=None, group: int = 0
 def make_schedule(kind: int, total_steps: int, max_lr: Sequence[float], weight_decay: Optional[Sequence[float]] = None,
                   pct_start: float = 0.3, div_factor: float = 25.0, final_div_factor: float = 1e4, autolr: int = 0,
                   warmup_steps: int = 0, beta: float = 0.9, sigma: float = 0.1, lambda_: float = 0.5,
-                  f_div: float = 25.0, f_final: float = 1.0) -> hdet_schedule:
+                  f_div: float = 25.0, f_final: float = 1.0, auto_wd: int = 0) -> hdet_schedule:
     s = hdet_schedule()
     s.kind, s.autolr, s.total_steps = kind, int(autolr), total_steps
     s._max_lr = _doubles(max_lr)            # keep the host arrays alive with the struct
@@ -174,6 +175,7 @@ def make_schedule(kind: int, total_steps: int, max_lr: Sequence[float], weight_d
     s.pct_start, s.div_factor, s.final_div_factor = pct_start, div_factor, final_div_factor
     s.warmup_steps, s.beta, s.sigma, s.lambda_ = warmup_steps, beta, sigma, lambda_
     s.f_div, s.f_final = f_div, f_final
+    s.auto_wd = int(auto_wd)
     return s
 
 

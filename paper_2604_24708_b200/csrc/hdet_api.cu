@@ -30,6 +30,9 @@ struct hdet_ctx {
   double ctrl_base[HDET_MAX_GROUPS]{};
   double velocity[HDET_MAX_GROUPS]{};
   double delta[HDET_MAX_GROUPS]{};
+  double wd_base[HDET_MAX_GROUPS]{};       // base weight decay per group (Remark 1 channel)
+  double wd_velocity[HDET_MAX_GROUPS]{};
+  double wd_delta[HDET_MAX_GROUPS]{};
   double lr[HDET_MAX_GROUPS][HDET_MAX_REPLICAS]{};
   double wd[HDET_MAX_GROUPS][HDET_MAX_REPLICAS]{};
   int32_t perm_lr[HDET_MAX_GROUPS][HDET_MAX_REPLICAS]{};
@@ -110,7 +113,7 @@ void compute_tables(hdet_ctx* h) {
     h->base[g] = b;
     for (int r = 0; r < n; ++r) {
       h->lr[g][r] = b * h->rho_lr[h->perm_lr[g][r]];
-      h->wd[g][r] = h->weight_decay[g] * h->rho_wd[h->perm_wd[g][r]];
+      h->wd[g][r] = h->wd_base[g] * h->rho_wd[h->perm_wd[g][r]];
     }
   }
 }
@@ -142,6 +145,9 @@ void export_state(const hdet_ctx* h, hdet_state* out) {
   std::memcpy(out->weights, h->weights, sizeof h->weights);
   std::memcpy(out->loss_acc, h->loss_acc, sizeof h->loss_acc);
   std::memcpy(out->loss_round, h->loss_round, sizeof h->loss_round);
+  std::memcpy(out->wd_base, h->wd_base, sizeof h->wd_base);
+  std::memcpy(out->wd_velocity, h->wd_velocity, sizeof h->wd_velocity);
+  std::memcpy(out->wd_delta, h->wd_delta, sizeof h->wd_delta);
   out->gamma = h->has_schedule ? decay_gamma(h->sched.f_div, h->sched.f_final, h->sched.total_steps,
                                              h->sched.warmup_steps, h->cfg.sync_interval)
                                : 0.0;
@@ -164,6 +170,9 @@ void import_state(hdet_ctx* h, const hdet_state* in) {
   std::memcpy(h->weights, in->weights, sizeof h->weights);
   std::memcpy(h->loss_acc, in->loss_acc, sizeof h->loss_acc);
   std::memcpy(h->loss_round, in->loss_round, sizeof h->loss_round);
+  std::memcpy(h->wd_base, in->wd_base, sizeof h->wd_base);
+  std::memcpy(h->wd_velocity, in->wd_velocity, sizeof h->wd_velocity);
+  std::memcpy(h->wd_delta, in->wd_delta, sizeof h->wd_delta);
 }
 
 DevConst device_constants(const hdet_ctx* h) {
@@ -173,6 +182,7 @@ DevConst device_constants(const hdet_ctx* h) {
   c.adam = h->cfg.optimizer == HDET_OPT_ADAMW;
   c.kind = h->sched.kind;
   c.autolr = h->sched.autolr;
+  c.auto_wd = h->sched.auto_wd;
   c.reshuffle = h->cfg.reshuffle;
   c.total_steps = h->sched.total_steps;
   c.warmup_steps = h->sched.warmup_steps;
@@ -362,6 +372,7 @@ int hdet_set_schedule(hdet_handle h, const hdet_schedule* s) {
   for (int g = 0; g < h->cfg.n_groups; ++g) {
     h->max_lr[g] = s->max_lr[g];
     h->weight_decay[g] = s->weight_decay ? s->weight_decay[g] : 0.0;
+    h->wd_base[g] = h->weight_decay[g];
   }
   h->sched.max_lr = nullptr;
   h->sched.weight_decay = nullptr;
@@ -599,6 +610,17 @@ int hdet_autolr_update(hdet_handle h, const double* round_losses, void* /*stream
     h->delta[g] = weighted - plain;                                        // Eq. 6
     h->velocity[g] = h->sched.beta * h->velocity[g] + (1.0 - h->sched.beta) * h->delta[g];   // Eq. 7
     h->ctrl_base[g] = plain * (1.0 - gamma) + h->velocity[g] * h->sched.lambda;
+    if (h->sched.auto_wd) {   // Remark 1: the same update on the weight decays of the last step, without decay
+      double w_wd = 0.0, p_wd = 0.0;
+      for (int r = 0; r < n; ++r) {
+        w_wd += h->weights[r] * h->wd[g][r];
+        p_wd += h->wd[g][r];
+      }
+      p_wd /= n;
+      h->wd_delta[g] = w_wd - p_wd;
+      h->wd_velocity[g] = h->sched.beta * h->wd_velocity[g] + (1.0 - h->sched.beta) * h->wd_delta[g];
+      h->wd_base[g] = p_wd + h->wd_velocity[g] * h->sched.lambda;
+    }
   }
   h->fired = true;
   if (h->cfg.reshuffle) {                                                   // Eq. 9
@@ -657,6 +679,9 @@ int hdet_set_state(hdet_handle h, const hdet_state* in) {
   }
   std::memcpy(h->loss_acc, in->loss_acc, sizeof h->loss_acc);
   std::memcpy(h->loss_round, in->loss_round, sizeof h->loss_round);
+  std::memcpy(h->wd_base, in->wd_base, sizeof h->wd_base);
+  std::memcpy(h->wd_velocity, in->wd_velocity, sizeof h->wd_velocity);
+  std::memcpy(h->wd[0], in->wd[0], sizeof h->wd);  // decays of the last update: the Remark 1 channel needs them at a round end
   h->device_mode = false;   // the host copy is authoritative again; hdet_step_device uploads it anew
   if (h->d_status) {
     DeviceScope scope(h->cfg.device);

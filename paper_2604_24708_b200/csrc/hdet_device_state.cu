@@ -37,7 +37,7 @@ __global__ void __launch_bounds__(32) device_scalars_kernel(DevState* d, const D
                                        c.final_div_factor);
     if (lane < c.n) {
       const double lr = b * spread_multiplier(c.n, c.alpha_lr, st.perm_lr[g][lane]);        // Eq. 1, Eq. 9
-      const double wd = c.weight_decay[g] * spread_multiplier(c.n, c.alpha_wd, st.perm_wd[g][lane]);
+      const double wd = st.wd_base[g] * spread_multiplier(c.n, c.alpha_wd, st.perm_wd[g][lane]);
       st.lr[g][lane] = lr;
       st.wd[g][lane] = wd;
       sc.lr_wd[g][lane] = (float)(c.adam ? lr * wd : wd);
@@ -97,6 +97,18 @@ __global__ void __launch_bounds__(32) device_round_end_kernel(DevState* d, const
       st.delta[g] = delta;
       st.velocity[g] = v;
       st.ctrl_base[g] = plain * (1.0 - gamma) + v * c.lambda;
+    }
+    if (c.auto_wd) {   // Remark 1: the same update on the weight decays of the last step, without decay
+      const double h = active ? st.wd[g][lane] : 0.0;
+      const double w_wd = warp_sum(w * h);
+      const double p_wd = warp_sum(h) / (double)c.n;
+      if (lane == 0) {
+        const double d_wd = w_wd - p_wd;
+        const double v_wd = c.ctrl_beta * st.wd_velocity[g] + (1.0 - c.ctrl_beta) * d_wd;
+        st.wd_delta[g] = d_wd;
+        st.wd_velocity[g] = v_wd;
+        st.wd_base[g] = p_wd + v_wd * c.lambda;
+      }
     }
   }
   if (lane == 0) st.fired = 1;

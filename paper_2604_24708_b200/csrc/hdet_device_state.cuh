@@ -9,7 +9,7 @@ namespace hdet {
 
 // Constants of a handle (configuration + schedule), passed by value to the scalar kernels.
 struct DevConst {
-  int n, n_groups, adam, kind, autolr, reshuffle;
+  int n, n_groups, adam, kind, autolr, auto_wd, reshuffle;
   long long total_steps, warmup_steps, sync_interval;
   double beta1, beta2, eps, momentum, alpha_lr, alpha_wd;
   double pct_start, div_factor, final_div_factor;

@@ -19,4 +19,4 @@ def schedule_for(w) -> B.hdet_schedule:
         w.sched_kind, w.total_steps, list(w.max_lr), list(w.weight_decay), pct_start=w.pct_start,
         div_factor=w.div_factor, final_div_factor=w.final_div_factor, autolr=w.autolr,
         warmup_steps=w.warmup_steps, beta=w.ctrl_beta, sigma=w.ctrl_sigma, lambda_=w.ctrl_lambda,
-        f_div=w.f_div, f_final=w.f_final)
+        f_div=w.f_div, f_final=w.f_final, auto_wd=getattr(w, "auto_wd", 0))

@@ -106,7 +106,7 @@ def oracle_for(w: W.Workload, params: Sequence[np.ndarray], groups: Sequence[int
         sync_interval=w.sync_interval, autolr=bool(w.autolr), warmup_steps=w.warmup_steps, ctrl_beta=w.ctrl_beta,
         ctrl_sigma=w.ctrl_sigma, ctrl_lambda=w.ctrl_lambda, f_div=w.f_div, f_final=w.f_final,
         reshuffle=bool(w.reshuffle), seed=w.seed, beta1=w.beta1, beta2=w.beta2, eps=w.eps, n_replicas=w.n_replicas,
-        grad_mean=grad_mean, momentum=w.momentum)
+        grad_mean=grad_mean, momentum=w.momentum, auto_wd=bool(w.auto_wd))
 
 
 class OracleRun:
@@ -209,6 +209,8 @@ def compare_scalars(st, o: O.HdetOracle, n: int, G: int, tol: float = 1e-12) -> 
         for r in range(n):
             close(st.lr[g][r], o.lr[g][r], f"lr[{g}][{r}]")
             close(st.wd[g][r], o.wd[g][r], f"wd[{g}][{r}]")
+        close(st.wd_base[g], o.wd_base[g], f"wd_base[{g}]")
+        assert abs(float(st.wd_velocity[g]) - o.vel_wd[g]) <= tol * max(abs(o.wd_base[g]), 1e-300), f"wd_velocity[{g}]"
         assert list(st.perm_lr[g])[:n] == o.perm_lr[g], f"perm_lr[{g}]"
         assert list(st.perm_wd[g])[:n] == o.perm_wd[g], f"perm_wd[{g}]"
     assert bool(st.fired) == o.fired

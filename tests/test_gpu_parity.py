@@ -255,6 +255,13 @@ def test_sgd_with_weight_decay_and_momentum_every_element(grad_dtype, align, mom
     _lockstep(w, H.whole_tensor_slabs(w), check_every=4, fuse=fuse, device_resident=True, grad_mean=True)
 
 
+@pytest.mark.parametrize("device_resident", [False, True])
+def test_weight_decay_channel_controller_every_element(device_resident):
+    """Remark 1: the controller also adapts the weight-decay base; host and device-resident stepping."""
+    w = replace(W.ragged_workload(n_replicas=5), auto_wd=1, total_steps=18)
+    _lockstep(w, H.whole_tensor_slabs(w), check_every=1, device_resident=device_resident)
+
+
 def test_alpha_zero_keeps_replicas_bitwise_identical():
     import torch
     w = replace(W.ragged_workload(n_replicas=6, numels=(4097, 33)), alpha_lr=0.0, alpha_wd=0.0, autolr=0)

@@ -214,6 +214,15 @@ def test_scalars_match_oracle_config3_and_config5():
     _scalar_run(W.ragged_workload())
 
 
+def test_scalars_match_oracle_with_the_weight_decay_channel_controller():
+    from dataclasses import replace
+    st, o, fired = _scalar_run(replace(W.config5(10), auto_wd=1))
+    assert fired == 90 and any(abs(st.wd_delta[g]) > 0 for g in (0, 2, 3))
+    assert st.wd_base[W.GROUP_NO_DECAY] == 0.0                      # a zero base stays zero
+    assert st.wd_base[0] != 0.05                                    # the base has moved
+    _scalar_run(replace(W.ragged_workload(), auto_wd=1))
+
+
 def test_mean_of_spread_rates_is_the_base_and_alpha_zero_is_uniform():
     w = W.config5(10)
     h = B.hdet_create(H.lib_config(B, w), [])
