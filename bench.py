@@ -284,19 +284,37 @@ def run_ours(args):
 
     # ---- end-to-end region: this step's gradients come from pinned host memory, the status word goes back --
     e2e_steps = max(1, min(args.steps, args.e2e_steps))
-    host_grad = torch.empty(arena.p_pad, dtype=arena.grad.dtype).pin_memory()
-    host_grad.copy_((arena.grad if args.shared_grad else arena.grad[0]).cpu())
     n_grad_copies = 1 if args.shared_grad else n
     h2d_bytes = n_grad_copies * arena.p_pad * arena.grad.element_size()
+    # Host stepping goes through hdet_step_host_grads: the library itself copies every tensor's gradients from a
+    # pinned host image of the gradient arena (same layout as on the device) and then launches the update.
+    host_image, host_ptrs, host_grad = None, None, None
+    if args.stepping == "host" and h2d_bytes <= (48 << 30):
+        try:
+            host_image = torch.empty(arena.grad.shape, dtype=arena.grad.dtype).pin_memory()
+            host_image.copy_(arena.grad)
+            gsz = arena.grad.element_size()
+            host_ptrs = [host_image.data_ptr() + gsz * off for off in arena.offsets]
+        except RuntimeError:
+            host_image = None
+    if host_image is None:
+        host_grad = torch.empty(arena.p_pad, dtype=arena.grad.dtype).pin_memory()
+        host_grad.copy_((arena.grad if args.shared_grad else arena.grad[0]).cpu())
 
     def e2e_step():
-        for r in range(n_grad_copies):
-            (arena.grad if args.shared_grad else arena.grad[r]).copy_(host_grad, non_blocking=True)
-        if args.stepping == "host":
-            one_step()
-        else:                                               # per step, so that every step sees its own gradients
-            B.hdet_step_device(h, d_losses[state["i"] % w.total_steps], stream.cuda_stream)
+        k = state["i"] % w.total_steps
+        if host_image is not None:
+            if B.hdet_step_host_grads(h, host_ptrs, losses[k], stream.cuda_stream):
+                B.hdet_autolr_update(h)
             state["i"] += 1
+        else:
+            for r in range(n_grad_copies):
+                (arena.grad if args.shared_grad else arena.grad[r]).copy_(host_grad, non_blocking=True)
+            if args.stepping == "host":
+                one_step()
+            else:                                           # per step, so that every step sees its own gradients
+                B.hdet_step_device(h, d_losses[k], stream.cuda_stream)
+                state["i"] += 1
         st = B.hdet_get_state(h, raise_on_nonfinite=False)   # reads the device status word back (synchronises)
         return st.device_status
 
@@ -383,8 +401,9 @@ def run_ours(args):
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d_bytes, "d2h_bytes_per_step": 4,
                 "steps": e2e_steps,
-                "what": "per step: gradients of all replicas copied from pinned host memory, hdet_step "
-                        "(+ hdet_autolr_update), device status word read back"},
+                "what": ("per step: hdet_step_host_grads copies the gradients of all replicas from pinned host memory "
+                         "and updates (+ hdet_autolr_update); device status word read back") if host_image is not None
+                else "per step: gradients copied from pinned host memory by the caller, then the step; status word read back"},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "traffic": traffic, "traffic_source": traffic_src, "peak_source": peak_src,
                      "kernel": ("fanout_shared_kernel" if args.shared_state else "fanout_kernel") + (" (fused update+converge)" if w.sync_interval == 1 else ""),

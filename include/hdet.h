@@ -210,6 +210,18 @@ HDET_API int hdet_set_schedule(hdet_handle h, const hdet_schedule* sched);
 HDET_API int hdet_step(hdet_handle h, const double* step_losses, void* stream, int32_t* did_converge);
 
 /*
+ * hdet_step_host_grads -- hdet_step for gradients that live in HOST memory: host_grads[k] points to
+ * the gradients of tensor k laid out like its device gradient (replica r at host_grads[k] +
+ * r * grad_stride elements; one copy when grad_stride is 0).  The call enqueues the host-to-device
+ * copies of all tensors on `stream` (one strided copy per tensor) and then the update, so the copies
+ * are inside the call.  The host buffers must stay valid until the stream has passed the copies; they
+ * should be pinned, otherwise every copy waits for the stream and stages through the driver.
+ * Errors: as hdet_step, plus INVALID_ARG for NULL pointers and CUDA for a failed copy.
+ */
+HDET_API int hdet_step_host_grads(hdet_handle h, const void* const* host_grads, const double* step_losses,
+                                  void* stream, int32_t* did_converge);
+
+/*
  * Replica axis sharded over GPUs (the paper's own arrangement, one or more replicas per GPU).
  * Every rank creates a handle with n_replicas = its local replicas, n_replicas_global = N and its
  * replica_offset, and per step:

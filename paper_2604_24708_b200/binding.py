@@ -93,6 +93,9 @@ def _load() -> C.CDLL:
     lib.hdet_step.argtypes = [H, C.POINTER(C.c_double), C.c_void_p, C.POINTER(C.c_int32)]
     lib.hdet_step_device.argtypes = [H, C.c_void_p, C.c_int32, C.c_void_p, C.POINTER(C.c_int32)]
     lib.hdet_step_device.restype = C.c_int
+    lib.hdet_step_host_grads.argtypes = [H, C.POINTER(C.c_void_p), C.POINTER(C.c_double), C.c_void_p,
+                                         C.POINTER(C.c_int32)]
+    lib.hdet_step_host_grads.restype = C.c_int
     lib.hdet_step_sharded.argtypes = [H, C.POINTER(C.c_double), C.c_void_p, C.c_void_p, C.POINTER(C.c_int32)]
     lib.hdet_step_sharded.restype = C.c_int
     lib.hdet_apply_mean.argtypes = [H, C.c_void_p, C.c_void_p]
@@ -209,6 +212,15 @@ def hdet_step_device(h, d_step_losses=None, stream: int = 0) -> bool:
         dtype = {torch.float32: HDET_DTYPE_F32, torch.float64: HDET_DTYPE_F64}[d_step_losses.dtype]
         ptr = C.c_void_p(d_step_losses.data_ptr())
     _check(_lib.hdet_step_device(h, ptr, dtype, C.c_void_p(stream), C.byref(flag)), h)
+    return bool(flag.value)
+
+
+def hdet_step_host_grads(h, host_grad_ptrs: Sequence[int], step_losses: Optional[Sequence[float]] = None,
+                         stream: int = 0) -> bool:
+    """hdet_step with the gradients taken from host memory (one pointer per tensor, laid out like the device gradient)."""
+    flag = C.c_int32(0)
+    arr = (C.c_void_p * max(1, len(host_grad_ptrs)))(*host_grad_ptrs) if host_grad_ptrs else None
+    _check(_lib.hdet_step_host_grads(h, arr, _doubles(step_losses), C.c_void_p(stream), C.byref(flag)), h)
     return bool(flag.value)
 
 

@@ -59,6 +59,7 @@ struct hdet_ctx {
   int r_offset = 0;            // global index of local replica 0
   int64_t partial_numel = 0;   // elements of the partial-sum staging buffer
   std::vector<int64_t> partial_offsets;  // per tensor, inside that buffer
+  std::vector<hdet_tensor> tensors;      // the caller's descriptors (for hdet_step_host_grads)
   int64_t launches = 0;
   std::string error;
 };
@@ -313,6 +314,7 @@ int hdet_create(const hdet_config* cfg, const hdet_tensor* tensors, int64_t n_te
   h->n_global = n_global;
   h->r_offset = sharded ? cfg->replica_offset : 0;
   h->partial_numel = partial_numel;
+  h->tensors.assign(tensors, tensors + n_tensors);
   for (const TensorDesc& d : descs) h->partial_offsets.push_back(d.partial_off);
   spread_multipliers(n_global, cfg->alpha_lr, h->rho_lr);
   spread_multipliers(n_global, cfg->alpha_wd, h->rho_wd);
@@ -455,6 +457,34 @@ static int step_impl(hdet_handle h, const double* step_losses, bool sharded_call
 }
 
 int hdet_step(hdet_handle h, const double* step_losses, void* stream, int32_t* did_converge) {
+  return step_impl(h, step_losses, false, nullptr, stream, did_converge);
+}
+
+int hdet_step_host_grads(hdet_handle h, const void* const* host_grads, const double* step_losses, void* stream,
+                         int32_t* did_converge) {
+  if (!h) return HDET_ERR_INVALID_ARG;
+  if (did_converge) *did_converge = 0;
+  if (h->n_tensors > 0 && !host_grads) return fail(h, HDET_ERR_INVALID_ARG, "hdet_step_host_grads: host_grads is NULL");
+  if (h->n_tensors > 0) {
+    DeviceScope scope(h->cfg.device);
+    if (scope.err != cudaSuccess) return fail_cuda(h, "hdet_step_host_grads", scope.err);
+    const size_t gsz = h->cfg.grad_dtype == HDET_DTYPE_BF16 ? 2 : 4;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    for (int64_t k = 0; k < h->n_tensors; ++k) {
+      const hdet_tensor& t = h->tensors[k];
+      if (!host_grads[k]) return fail(h, HDET_ERR_INVALID_ARG, "hdet_step_host_grads: a host gradient pointer is NULL");
+      const size_t row = (size_t)t.numel * gsz;
+      cudaError_t e;
+      if (t.grad_stride == 0 || h->cfg.n_replicas == 1) {
+        e = cudaMemcpyAsync(t.grad, host_grads[k], row, cudaMemcpyHostToDevice, st);
+      } else {   // N rows of one tensor, replica stride as pitch on both sides
+        const size_t pitch = (size_t)t.grad_stride * gsz;
+        e = cudaMemcpy2DAsync(t.grad, pitch, host_grads[k], pitch, row, (size_t)h->cfg.n_replicas,
+                              cudaMemcpyHostToDevice, st);
+      }
+      if (e != cudaSuccess) return fail_cuda(h, "hdet_step_host_grads: gradient upload", e);
+    }
+  }
   return step_impl(h, step_losses, false, nullptr, stream, did_converge);
 }
 

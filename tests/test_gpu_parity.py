@@ -450,3 +450,28 @@ def test_warm_noisy_init_config2_statistics_and_sampled_parity():
         got = after[:, offs[k] + s0:offs[k] + s0 + ln]
         assert H.rel_err(got, ref).max() <= TOL_ONE_STEP
     g.close()
+
+
+def test_step_with_host_gradients_equals_step_with_device_gradients():
+    """hdet_step_host_grads: the library uploads each tensor's gradients (strided per replica), then updates."""
+    import torch
+    for shared in (False, True):
+        w = W.ragged_workload(n_replicas=4, numels=(4099, 7, 2048, 33))
+        ref, _ = _final_arena(w, shared_grad=shared, steps=6)
+        g = H.GpuRun(w, shared_grad=shared)
+        gsz = g.arena.grad.element_size()
+        for i in range(6):
+            g.fill_grads(i)
+            host = g.arena.grad.cpu().pin_memory()
+            g.arena.grad.zero_()                               # the device copy must come from the host image
+            ptrs = [host.data_ptr() + gsz * off for off in g.arena.offsets]
+            losses = list(R.step_losses(w, i, g.perm0()))
+            if g.B.hdet_step_host_grads(g.h, ptrs, losses):
+                g.B.hdet_autolr_update(g.h)
+            torch.cuda.synchronize()
+            g.i += 1
+        for a, b in zip(ref, [g.arena.param, g.arena.exp_avg, g.arena.exp_avg_sq]):
+            assert torch.equal(a, b)
+        with pytest.raises(g.B.HdetError):
+            g.B.hdet_step_host_grads(g.h, [0] * len(w.tensors), None)
+        g.close()
