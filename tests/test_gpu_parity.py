@@ -475,3 +475,11 @@ def test_step_with_host_gradients_equals_step_with_device_gradients():
         with pytest.raises(g.B.HdetError):
             g.B.hdet_step_host_grads(g.h, [0] * len(w.tensors), None)
         g.close()
+
+
+def test_maximum_replicas_and_groups():
+    """N = 32 replicas and G = 8 groups: every slot of the 8 x 32 launch-scalar tables is in use."""
+    w = W.ragged_workload(n_replicas=32, n_groups=8, numels=(2051, 7, 4096, 33, 1, 2048, 515, 9, 130, 4100))
+    w = replace(w, total_steps=9, warmup_steps=3)
+    _lockstep(w, H.whole_tensor_slabs(w), check_every=3)
+    _lockstep(w, H.whole_tensor_slabs(w), check_every=3, device_resident=True)
