@@ -69,18 +69,25 @@ __device__ __forceinline__ void gaussian_pair(unsigned long long key, unsigned l
   const unsigned long long u = mix64(key + p * kGolden);
   const float u1 = ((float)(unsigned)(u >> 41) + 0.5f) * (1.0f / 8388608.0f);
   const float u2 = (float)(unsigned)((u >> 16) & 0xFFFFFFull) * (1.0f / 16777216.0f);
+  // logf stays exact-rounded (u1 can be within 2^-24 of 1, where a fast log would lose the radius);
+  // sine and cosine use the fast intrinsics on an angle reduced to [-pi, pi): cos(a + pi) = -cos a.
   const float radius = sqrtf(-2.0f * logf(u1));
   float s, c;
-  sincospif(2.0f * u2, &s, &c);
-  z_even = radius * c;
-  z_odd = radius * s;
+  __sincosf(6.283185307179586f * (u2 - 0.5f), &s, &c);
+  z_even = -radius * c;
+  z_odd = -radius * s;
 }
 
 __global__ void __launch_bounds__(kThreads, 4)
 warm_noise_kernel(const __grid_constant__ LaunchPlan plan, const double* sigma_ptr, int n, unsigned long long base_key) {
   const float sigma = (float)(*sigma_ptr);
+  __shared__ unsigned long long keys[HDET_MAX_REPLICAS];   // one key per replica for the tile's tensor
   for (int t = blockIdx.x; t < plan.n_tiles; t += gridDim.x) {
     const Tile tile = plan.tiles[t];
+    __syncthreads();
+    if (threadIdx.x < n)
+      keys[threadIdx.x] = mix64(mix64(base_key + (unsigned long long)threadIdx.x) + (unsigned long long)tile.tensor);
+    __syncthreads();
     const TensorDesc td = plan.tensors[tile.tensor];
     const long long off = (long long)tile.tile * kTileElems;
     const long long rest = td.numel - off;
@@ -91,7 +98,7 @@ warm_noise_kernel(const __grid_constant__ LaunchPlan plan, const double* sigma_p
       const float4 x0 = __ldcs(reinterpret_cast<const float4*>(P + 4 * j));       // checkpoint, read once
       const unsigned long long p = (unsigned long long)(off + 4 * j) >> 1;        // first of two element pairs
       for (int r = 0; r < n; ++r) {
-        const unsigned long long key = mix64(mix64(base_key + (unsigned long long)r) + (unsigned long long)tile.tensor);
+        const unsigned long long key = keys[r];
         float z0, z1, z2, z3;
         gaussian_pair(key, p, z0, z1);
         gaussian_pair(key, p + 1, z2, z3);
@@ -103,7 +110,7 @@ warm_noise_kernel(const __grid_constant__ LaunchPlan plan, const double* sigma_p
       const float x0 = __ldcs(P + e);
       const unsigned long long elem = (unsigned long long)(off + e);
       for (int r = 0; r < n; ++r) {
-        const unsigned long long key = mix64(mix64(base_key + (unsigned long long)r) + (unsigned long long)tile.tensor);
+        const unsigned long long key = keys[r];
         float ze, zo;
         gaussian_pair(key, elem >> 1, ze, zo);
         __stcs(P + r * td.param_stride + e, fmaf(sigma, (elem & 1) ? zo : ze, x0));
