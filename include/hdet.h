@@ -13,6 +13,12 @@
  *   hdet_autolr_update controller (Eq. 4 - Eq. 9) after a converge
  *   hdet_get_state / hdet_set_state   scalars for logging and resume
  *   hdet_destroy
+ * and, around that core:
+ *   hdet_step_device       the same step with the scalar state and the controller on the device
+ *   hdet_step_host_grads   the same step with the gradients uploaded from host memory first
+ *   hdet_step_sharded / hdet_apply_mean / hdet_partial_layout   replica axis split over GPUs
+ *   hdet_warm_init         warm noisy initialisation (Eq. 10)
+ *   hdet_converge_static   allocation-free variant of hdet_converge
  *
  * Conventions
  *   - Every tensor pointer is a DEVICE pointer owned by the caller; it must stay
@@ -26,8 +32,9 @@
  *     on the device by the caller (same stream, or events).
  *   - No function throws or aborts; each returns an hdet_status.  hdet_last_error
  *     gives a text for the last failure on a handle.
- *   - The library owns only its work table, a status word on the device and the host
- *     controller state.  hdet_step / hdet_converge / hdet_autolr_update allocate nothing.
+ *   - The library owns only its work table, a status word and a small state block on the
+ *     device, and the host controller state.  hdet_step / hdet_step_device / hdet_converge /
+ *     hdet_autolr_update allocate nothing.
  *   - There is no CPU fallback: a handle with tensors needs a CUDA device.  A handle
  *     created with n_tensors == 0 touches no device and runs only the scalar part
  *     (schedule, spread, controller), which is what host-side tests use.
