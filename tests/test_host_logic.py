@@ -267,3 +267,26 @@ def test_state_roundtrip_resumes_identically():
     assert e.value.status == B.HDET_ERR_INVALID_ARG
     B.hdet_destroy(a)
     B.hdet_destroy(b)
+
+
+def test_binding_fails_loudly_without_the_library(monkeypatch, tmp_path):
+    """No CPU fallback: a missing libhdet.so is an import error, not a silent slow path."""
+    monkeypatch.setattr(B, "LIB_PATH", str(tmp_path / "libhdet.so"))
+    with pytest.raises(ImportError) as e:
+        B._load()
+    assert "no CPU fallback" in str(e.value)
+
+
+def test_arena_refuses_to_run_without_a_device():
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a CUDA device is present")
+    from paper_2604_24708_b200.arena import StackedArena
+    with pytest.raises(RuntimeError):
+        StackedArena([8], [0], 2, B.HDET_OPT_SGD, B.HDET_DTYPE_F32)
+    # and a handle with tensors cannot be created without a device: the library reports the CUDA error
+    t = B.hdet_tensor(param=0x1000, grad=0x2000, numel=8, param_stride=8, grad_stride=8, state_stride=8, group=0)
+    cfg = _cfg(optimizer=B.HDET_OPT_SGD, grad_dtype=B.HDET_DTYPE_F32)
+    with pytest.raises(B.HdetError) as e:
+        B.hdet_create(cfg, [t])
+    assert e.value.status == B.HDET_ERR_CUDA
