@@ -64,7 +64,9 @@ typedef enum {
   HDET_ERR_ALIGN = 3,       /* a pointer is not aligned to its element type              */
   HDET_ERR_UNSUPPORTED = 4, /* a valid request this build does not implement             */
   HDET_ERR_CUDA = 5,        /* a CUDA runtime call failed; see hdet_last_error           */
-  HDET_ERR_NONFINITE = 6    /* a kernel produced a non-finite parameter (sticky)         */
+  HDET_ERR_NONFINITE = 6,   /* a kernel produced a non-finite parameter (sticky)         */
+  HDET_ERR_TIMEOUT = 7      /* a kernel gave up waiting for one of its own bulk copies and
+                               left a tile unfinished (sticky; parameters are then undefined) */
 } hdet_status;
 
 enum { HDET_OPT_SGD = 0, HDET_OPT_ADAMW = 1 };
@@ -155,7 +157,8 @@ typedef struct {
   int32_t fired;                      /* the controller has taken over the base rate       */
   int32_t round_ended;                /* the last hdet_step ended a round and
                                          hdet_autolr_update has not run since             */
-  uint32_t device_status;             /* bit 0: a non-finite parameter was produced        */
+  uint32_t device_status;             /* bit 0: a non-finite parameter was produced;
+                                         bit 1: a bounded wait inside a kernel ran out     */
   int32_t reserved;
   double base[HDET_MAX_GROUPS];       /* base rate used by the last update                 */
   double ctrl_base[HDET_MAX_GROUPS];  /* eta_bar held by the controller (Eq. 7)            */
@@ -191,11 +194,14 @@ HDET_API int hdet_create(const hdet_config* cfg, const hdet_tensor* tensors, int
  * hdet_set_schedule -- stores the base schedule eta(t) named in Algorithm 1's Require
  * list (one-cycle policy with cosine or linear annealing, or a constant) and the
  * controller constants (beta, sigma, lambda of Eq. 4 / Eq. 7; f_div, f_final of Eq. 8;
- * S_warm).  May be called again at any time; it does not reset the step count, but it
- * resets the base weight decays to sched->weight_decay.
+ * S_warm).  May be called again while the handle steps on the host; it does not reset the step
+ * count, but it resets the base weight decays to sched->weight_decay.  While the scalar state
+ * lives on the device (after hdet_step_device) the call returns HDET_ERR_STATE and changes
+ * nothing: a schedule change would reach only part of the device state.  hdet_get_state followed
+ * by hdet_set_state returns the handle to host stepping, where the schedule can be replaced.
  * Updates past step S keep the rate of step S - 1.
  * Errors: INVALID_ARG (NULL, S < 1, max_lr NULL, p*S <= 1 or p >= 1 for a one-cycle
- * kind, factors <= 0, sigma <= 0 with autolr, f_div or f_final <= 0).
+ * kind, factors <= 0, sigma <= 0 with autolr, f_div or f_final <= 0), STATE (device-resident stepping).
  */
 HDET_API int hdet_set_schedule(hdet_handle h, const hdet_schedule* sched);
 
@@ -316,7 +322,10 @@ HDET_API int hdet_autolr_update(hdet_handle h, const double* round_losses, void*
 /*
  * hdet_get_state -- copies the scalar state into *out.  Reads the device status word,
  * which synchronises with the device (cudaMemcpy) when the handle has tensors.
- * Returns HDET_ERR_NONFINITE (with *out filled) if a kernel flagged a non-finite value.
+ * Returns HDET_ERR_NONFINITE (with *out filled) if a kernel flagged a non-finite value, and
+ * HDET_ERR_TIMEOUT (with *out filled) if a kernel's bounded wait for its own copies ran out: the
+ * kernels never spin without a limit, so a copy that does not complete ends as this status instead
+ * of a hang.
  */
 HDET_API int hdet_get_state(hdet_handle h, hdet_state* out);
 
@@ -351,13 +360,15 @@ HDET_API int hdet_destroy(hdet_handle h);
  * should use hdet_converge.
  *
  * The first call on a device resolves the array's device address (cudaGetSymbolAddress) and
- * queries the launch shape; make that first call outside any stream capture.  All calls share the
- * array, which keeps the previous call's contents: each call clears the status word and rewrites
- * the tables it uses, in stream order.  Two calls whose work overlaps on the GPU (different
- * streams without an event between them, or different host threads) race on the array and must
- * be serialised by the caller.  The copies of the tables come from pageable host memory, so the
- * call may wait for earlier work on `stream`.
- * Errors: INVALID_ARG, ALIGN, UNSUPPORTED (limits), CUDA; text via hdet_last_error(NULL).
+ * queries the launch shape; make that first call before any stream capture begins.  All calls share
+ * the array, which keeps the previous call's contents: nothing in it has to start at zero, and each
+ * call rewrites the tables it is going to read, in stream order.  Two calls whose work overlaps on the
+ * GPU (different streams without an event between them, or different host threads) race on the array
+ * and must be serialised by the caller.  The tables are copied from temporary pageable host memory
+ * on every call, so the call may wait for earlier work on `stream`, and a call on a stream that is
+ * being captured is refused with HDET_ERR_UNSUPPORTED (a recorded copy would outlive its source).
+ * A non-finite mean is not reported by this entry point (it has no handle to hold a status).
+ * Errors: INVALID_ARG, ALIGN, UNSUPPORTED (limits, capturing stream), CUDA; text via hdet_last_error(NULL).
  */
 #define HDET_STATIC_MAX_TENSORS 1024
 #define HDET_STATIC_MAX_TILES 65536

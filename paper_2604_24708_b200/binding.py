@@ -19,6 +19,7 @@ HDET_ERR_ALIGN = 3
 HDET_ERR_UNSUPPORTED = 4
 HDET_ERR_CUDA = 5
 HDET_ERR_NONFINITE = 6
+HDET_ERR_TIMEOUT = 7
 
 HDET_OPT_SGD, HDET_OPT_ADAMW = 0, 1
 HDET_DTYPE_F32, HDET_DTYPE_BF16, HDET_DTYPE_F64 = 0, 1, 2

@@ -293,7 +293,9 @@ int hdet_create(const hdet_config* cfg, const hdet_tensor* tensors, int64_t n_te
     if (cfg->optimizer == HDET_OPT_ADAMW)
       vec = vec && aligned(t.exp_avg, 16) && aligned(t.exp_avg_sq, 16) && t.state_stride % 4 == 0;
     if (sgd_momentum) vec = vec && aligned(t.exp_avg, 16) && t.state_stride % 4 == 0;
-    d.vec = vec ? 1 : 0;
+    d.vec = vec ? kVecLoads : 0;
+    // Bulk copies move whole tiles and need every array, the gradient included, on 16-byte boundaries.
+    if (vec && adamw && aligned(t.grad, 16) && (t.grad_stride * (int64_t)gsz) % 16 == 0) d.vec |= kVecBulk;
     d.partial_off = partial_numel;
     d.partial = nullptr;
     partial_numel += (t.numel + 3) / 4 * 4;
@@ -349,6 +351,9 @@ int hdet_create(const hdet_config* cfg, const hdet_tensor* tensors, int64_t n_te
 int hdet_set_schedule(hdet_handle h, const hdet_schedule* s) {
   if (!h) return HDET_ERR_INVALID_ARG;
   if (!s || !s->max_lr) return fail(h, HDET_ERR_INVALID_ARG, "hdet_set_schedule: sched and max_lr must not be NULL");
+  if (h->device_mode)
+    return fail(h, HDET_ERR_STATE, "hdet_set_schedule: the scalar state lives on the device; hdet_get_state then "
+                                   "hdet_set_state returns the handle to host stepping, where the schedule can be replaced");
   if (s->kind < HDET_SCHED_CONSTANT || s->kind > HDET_SCHED_ONECYCLE_LINEAR)
     return fail(h, HDET_ERR_INVALID_ARG, "hdet_set_schedule: unknown kind");
   if (s->total_steps < 1) return fail(h, HDET_ERR_INVALID_ARG, "hdet_set_schedule: total_steps must be >= 1");
@@ -549,7 +554,7 @@ int hdet_step_device(hdet_handle h, const void* d_step_losses, int32_t loss_dtyp
   if (e != cudaSuccess) return fail_cuda(h, "hdet_step_device: scalar kernel launch", e);
   ++h->launches;
   const bool fuse = ends_round && h->cfg.fuse_converge;
-  LaunchPlan plan{h->d_tensors, h->d_tiles, h->n_tiles, h->grid_fanout, h->d_status, &h->d_state->scal};
+  LaunchPlan plan{h->d_tensors, h->d_tiles, h->n_tiles, h->grid_fanout, h->d_status, &h->d_state->scal, nullptr};
   const StepScalars unused{};
   e = launch_fanout(h->cfg.optimizer, h->cfg.optimizer == HDET_OPT_SGD && h->cfg.momentum != 0.0, h->cfg.grad_dtype, fuse,
                                   h->cfg.grad_mode == HDET_GRAD_REPLICA_MEAN,
@@ -683,6 +688,7 @@ int hdet_get_state(hdet_handle h, hdet_state* out) {
     if (e == cudaSuccess) e = cudaMemcpy(&word, h->d_status, sizeof word, cudaMemcpyDeviceToHost);
     if (e != cudaSuccess) return fail_cuda(h, "hdet_get_state", e);
     out->device_status = word;
+    if (word & 2u) return fail(h, HDET_ERR_TIMEOUT, "a kernel's bounded wait for its own bulk copies ran out; a tile was left unfinished");
     if (word & 1u) return fail(h, HDET_ERR_NONFINITE, "a kernel produced a non-finite parameter");
   }
   return HDET_OK;

@@ -13,6 +13,10 @@ constexpr int kThreads = 256;
 constexpr int kTileVecs = 2;
 constexpr int kTileElems = kThreads * 4 * kTileVecs;  // 2048 elements
 
+// Bits of TensorDesc::vec.
+constexpr int kVecLoads = 1;
+constexpr int kVecBulk = 2;
+
 // Per-tensor descriptor, resident on the device (built once by hdet_create).
 struct TensorDesc {
   float* param;
@@ -24,7 +28,7 @@ struct TensorDesc {
   long long grad_stride;
   long long state_stride;  // 0: one pair of moments shared by all replicas
   int group;
-  int vec;  // 1: pointers and strides allow 128-bit accesses
+  int vec;  // kVecLoads: pointers and strides allow 128-bit accesses; | kVecBulk: also 16-byte bulk copies of whole tiles
   long long partial_off;  // element offset of this tensor inside the partial-sum staging buffer (multiple of 4)
   float* partial;         // set per tile by the kernels (NULL in the table)
 };
@@ -46,6 +50,32 @@ struct StepScalars {
   double inv_n;     // 1 / N
   int n_replicas;
 };
+
+// Eq. 3 on one tile: every replica <- (1/N) sum over replicas, fp64 accumulation r = 0..N-1, one rounding.
+// The one statement of the stand-alone mean; hdet_converge and hdet_converge_static both run it.
+__device__ __forceinline__ void converge_tile(const TensorDesc& td, int tile_index, int n, double inv_n) {
+  const long long off = (long long)tile_index * kTileElems;
+  const long long rest = td.numel - off;
+  const int len = rest < kTileElems ? (int)rest : kTileElems;
+  const int nvec = td.vec ? (len >> 2) : 0;
+  float* const P = td.param + off;
+  for (int j = threadIdx.x; j < nvec; j += kThreads) {
+    double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
+#pragma unroll 4
+    for (int r = 0; r < n; ++r) {
+      const float4 x = __ldcs(reinterpret_cast<const float4*>(P + r * td.param_stride + 4 * j));
+      s0 += (double)x.x; s1 += (double)x.y; s2 += (double)x.z; s3 += (double)x.w;
+    }
+    const float4 mean = make_float4((float)(s0 * inv_n), (float)(s1 * inv_n), (float)(s2 * inv_n), (float)(s3 * inv_n));
+    for (int r = 0; r < n; ++r) __stcs(reinterpret_cast<float4*>(P + r * td.param_stride + 4 * j), mean);
+  }
+  for (int e = 4 * nvec + threadIdx.x; e < len; e += kThreads) {
+    double sum = 0.0;
+    for (int r = 0; r < n; ++r) sum += (double)__ldcs(P + r * td.param_stride + e);
+    const float mean = (float)(sum * inv_n);
+    for (int r = 0; r < n; ++r) __stcs(P + r * td.param_stride + e, mean);
+  }
+}
 
 struct LaunchPlan {
   const TensorDesc* tensors;

@@ -18,52 +18,26 @@ using hdet::Tile;
 constexpr int kMaxTensors = HDET_STATIC_MAX_TENSORS;
 constexpr int kMaxTiles = HDET_STATIC_MAX_TILES;
 
-// Layout of the scratch array: [status word, padded to 256 B][tensor descriptors][tiles].
-constexpr size_t kStatusBytes = 256;
+// Layout of the scratch array: [tensor descriptors][tiles].  Nothing in it has to start at zero: a call
+// overwrites every entry it is going to read.
 constexpr size_t kDescBytes = sizeof(TensorDesc) * kMaxTensors;
 constexpr size_t kTileBytes = sizeof(Tile) * kMaxTiles;
-constexpr size_t kScratchBytes = kStatusBytes + kDescBytes + kTileBytes;   // about 0.6 MB per GPU
+constexpr size_t kScratchBytes = kDescBytes + kTileBytes;   // about 0.6 MB per GPU
 
 // Every GPU that loads the library holds this array until the process exits.  In host code the
 // name `g_scratch` is only a handle for the runtime, not a device address: the address a kernel
 // can use comes from cudaGetSymbolAddress (see scratch_for_device below).
 static __device__ __align__(256) unsigned char g_scratch[kScratchBytes];
 
-__device__ __forceinline__ bool not_finite(float x) { return !(fabsf(x) <= 3.402823466e38f); }
-
+// The arithmetic is hdet::converge_tile, the same device function hdet_converge runs.
 __global__ void __launch_bounds__(kThreads, 4)
 converge_static_kernel(const TensorDesc* __restrict__ tensors, const Tile* __restrict__ tiles, int n_tiles, int n,
                        double inv_n) {
-  bool bad = false;
   for (int t = blockIdx.x; t < n_tiles; t += gridDim.x) {
     const Tile tile = tiles[t];
     const TensorDesc td = tensors[tile.tensor];
-    const long long off = (long long)tile.tile * kTileElems;
-    const long long rest = td.numel - off;
-    const int len = rest < kTileElems ? (int)rest : kTileElems;
-    const int nvec = td.vec ? (len >> 2) : 0;
-    float* const P = td.param + off;
-    for (int j = threadIdx.x; j < nvec; j += kThreads) {
-      double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
-#pragma unroll 4
-      for (int r = 0; r < n; ++r) {
-        const float4 x = __ldcs(reinterpret_cast<const float4*>(P + r * td.param_stride + 4 * j));
-        s0 += (double)x.x; s1 += (double)x.y; s2 += (double)x.z; s3 += (double)x.w;
-      }
-      const float4 mean = make_float4((float)(s0 * inv_n), (float)(s1 * inv_n), (float)(s2 * inv_n), (float)(s3 * inv_n));
-      bad |= not_finite(mean.x) || not_finite(mean.y) || not_finite(mean.z) || not_finite(mean.w);
-      for (int r = 0; r < n; ++r) __stcs(reinterpret_cast<float4*>(P + r * td.param_stride + 4 * j), mean);
-    }
-    for (int e = 4 * nvec + threadIdx.x; e < len; e += kThreads) {
-      double sum = 0.0;
-      for (int r = 0; r < n; ++r) sum += (double)__ldcs(P + r * td.param_stride + e);
-      const float mean = (float)(sum * inv_n);
-      bad |= not_finite(mean);
-      for (int r = 0; r < n; ++r) __stcs(P + r * td.param_stride + e, mean);
-    }
+    hdet::converge_tile(td, tile.tile, n, inv_n);
   }
-  // Device code may name the array directly: word 0 is the status word (bit 0 = non-finite mean).
-  if (bad) atomicOr(reinterpret_cast<unsigned*>(g_scratch), 1u);
 }
 
 struct DeviceSetup {
@@ -143,7 +117,7 @@ extern "C" HDET_API int hdet_converge_static(const hdet_tensor* tensors, int64_t
     d.param = static_cast<float*>(t.param);
     d.numel = t.numel;
     d.param_stride = t.param_stride;
-    d.vec = (reinterpret_cast<uintptr_t>(t.param) % 16 == 0 && t.param_stride % 4 == 0) ? 1 : 0;
+    d.vec = (reinterpret_cast<uintptr_t>(t.param) % 16 == 0 && t.param_stride % 4 == 0) ? hdet::kVecLoads : 0;
     descs[k] = d;
   }
   tiles.reserve(total_tiles);
@@ -154,17 +128,23 @@ extern "C" HDET_API int hdet_converge_static(const hdet_tensor* tensors, int64_t
   int prev = -1;
   cudaError_t e = cudaGetDevice(&prev);
   if (e == cudaSuccess && prev != device) e = cudaSetDevice(device);
-  DeviceSetup* setup = nullptr;
-  if (e == cudaSuccess) e = scratch_for_device(device, &setup);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // The tables are copied from host buffers that die with this call, so the call cannot be recorded
+  // into a stream capture: a replay would read freed host memory.  Refuse instead.
+  bool capturing = false;
   if (e == cudaSuccess) {
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    e = cudaStreamIsCapturing(st, &cap);
+    capturing = e == cudaSuccess && cap != cudaStreamCaptureStatusNone;
+  }
+  DeviceSetup* setup = nullptr;
+  if (e == cudaSuccess && !capturing) e = scratch_for_device(device, &setup);
+  if (e == cudaSuccess && !capturing) {
     unsigned char* base = setup->scratch;
-    TensorDesc* d_desc = reinterpret_cast<TensorDesc*>(base + kStatusBytes);
-    Tile* d_tiles = reinterpret_cast<Tile*>(base + kStatusBytes + kDescBytes);
-    // The array keeps the previous call's contents: clear the status word, overwrite the tables in use.
-    e = cudaMemsetAsync(base, 0, kStatusBytes, st);
-    if (e == cudaSuccess)
-      e = cudaMemcpyAsync(d_desc, descs.data(), descs.size() * sizeof(TensorDesc), cudaMemcpyHostToDevice, st);
+    TensorDesc* d_desc = reinterpret_cast<TensorDesc*>(base);
+    Tile* d_tiles = reinterpret_cast<Tile*>(base + kDescBytes);
+    // The array keeps the previous call's contents: overwrite the tables this call uses, in stream order.
+    e = cudaMemcpyAsync(d_desc, descs.data(), descs.size() * sizeof(TensorDesc), cudaMemcpyHostToDevice, st);
     if (e == cudaSuccess)
       e = cudaMemcpyAsync(d_tiles, tiles.data(), tiles.size() * sizeof(Tile), cudaMemcpyHostToDevice, st);
     if (e == cudaSuccess) {
@@ -175,6 +155,9 @@ extern "C" HDET_API int hdet_converge_static(const hdet_tensor* tensors, int64_t
     }
   }
   if (prev >= 0 && prev != device) cudaSetDevice(prev);
+  if (capturing)
+    return fail(HDET_ERR_UNSUPPORTED, "hdet_converge_static: the stream is being captured; this call copies its tables "
+                                      "from temporary host memory and refuses to be recorded");
   if (e != cudaSuccess) {
     char msg[200];
     snprintf(msg, sizeof msg, "hdet_converge_static: %s", cudaGetErrorString(e));

@@ -71,9 +71,11 @@ def test_config1_sgd_every_element_every_step():
 
 @pytest.mark.parametrize("optimizer,grad_dtype", [(W.OPT_ADAMW, W.DTYPE_BF16), (W.OPT_ADAMW, W.DTYPE_F32),
                                                    (W.OPT_SGD, W.DTYPE_F32), (W.OPT_SGD, W.DTYPE_BF16)])
-@pytest.mark.parametrize("align", [8, 1])
+@pytest.mark.parametrize("align", [8, 4, 1])
 def test_ragged_list_every_element(optimizer, grad_dtype, align):
-    """Odd sizes: tails shorter than a vector, exact tile multiples, one element; align=1 forces scalar accesses."""
+    """Odd sizes: tails shorter than a vector, exact tile multiples, one element.  align=8: bulk copies for full
+    tiles; align=4: bf16 gradients are then only 8-byte aligned, so 128-bit loads without bulk copies; align=1
+    forces scalar accesses."""
     w = W.ragged_workload(n_replicas=3, optimizer=optimizer, grad_dtype=grad_dtype, align_elems=align)
     _lockstep(w, H.whole_tensor_slabs(w), check_every=1)
 
@@ -117,7 +119,7 @@ def test_fused_converge_equals_update_then_converge_bitwise_and_runs_are_determi
 
 @pytest.mark.parametrize("optimizer,grad_dtype", [(W.OPT_ADAMW, W.DTYPE_BF16), (W.OPT_ADAMW, W.DTYPE_F32),
                                                    (W.OPT_SGD, W.DTYPE_F32), (W.OPT_SGD, W.DTYPE_BF16)])
-@pytest.mark.parametrize("align", [8, 1])
+@pytest.mark.parametrize("align", [8, 4, 1])
 def test_gradient_replica_mean_every_element(optimizer, grad_dtype, align):
     """grad_mode = replica mean (Algorithm 1's gradient all-reduce on the device), per-replica moments."""
     w = W.ragged_workload(n_replicas=5, optimizer=optimizer, grad_dtype=grad_dtype, align_elems=align)
@@ -187,9 +189,15 @@ def test_device_resident_equals_host_stepping_and_mode_switches():
     with pytest.raises(g.B.HdetError) as e:
         g.B.hdet_autolr_update(g.h)
     assert e.value.status == g.B.HDET_ERR_STATE
+    # a schedule change would reach only part of the device-resident state: refused until the state is back on the host
+    with pytest.raises(g.B.HdetError) as e:
+        g.B.hdet_set_schedule(g.h, H.lib_schedule(g.B, w))
+    assert e.value.status == g.B.HDET_ERR_STATE
     st = g.state()
     assert st.step == 5
     g.B.hdet_set_state(g.h, st)
+    g.B.hdet_set_schedule(g.h, H.lib_schedule(g.B, w))       # accepted again (same schedule: the run continues unchanged)
+    g.B.hdet_set_state(g.h, st)                               # the call reset the base weight decays; restore them
     g.device_resident = False
     for i in range(5, w.total_steps):
         g.step(g.perm0())
@@ -328,6 +336,25 @@ def test_nonfinite_parameter_sets_the_status_word():
     g.B.hdet_set_state(g.h, st)            # clears the word
     assert g.B.hdet_get_state(g.h).device_status == 0
     g.close()
+
+
+@pytest.mark.parametrize("align", [8, 4])
+def test_eps_zero_on_a_ragged_list_sets_no_status_bit(align):
+    """eps = 0 is accepted.  Idle lanes of a partial tile hold zeros and would compute 0/0 there; that must
+    neither reach memory nor the status word."""
+    w = replace(W.ragged_workload(n_replicas=3, align_elems=align), eps=0.0)
+    slabs = H.whole_tensor_slabs(w)
+    o = H.OracleRun(w, slabs)
+    # precondition of the case: no first gradient is exactly zero (v would stay 0 and 0/0 would be genuine)
+    assert all(np.all(g != 0.0) for g in o.grads(0))
+    g = H.GpuRun(w)
+    try:
+        for i in range(3):
+            assert g.step(g.perm0()) == o.step()
+            H.compare_slabs(g, o, TOL_ONE_STEP if i == 0 else TOL_FULL_RUN)
+            assert g.state().device_status == 0
+    finally:
+        g.close()
 
 
 def test_config2_full_run_sampled():

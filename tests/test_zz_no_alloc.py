@@ -67,7 +67,7 @@ def test_static_converge_matches_the_handle_entry_point_on_two_calls_in_a_row():
     # first call: a long ragged list (vector path, tails); second call: a shorter list with odd
     # offsets (scalar path) and another replica count, so stale tables from call 1 would show.
     first = make([4099, 2048, 3, 70001, 1, 12289], 8, 1, 8)
-    second = make([5, 2051, 33], 3, 2, 1)
+    second = make([5, 2051, 33, 6151], 3, 2, 1)      # 6151 elements: four tiles on the scalar path
     before_first = first.param.double().cpu().numpy()
     want_first, want_second = reference(first, 8, 8), reference(second, 3, 1)
     stream = torch.cuda.current_stream().cuda_stream
@@ -91,3 +91,20 @@ def test_static_converge_matches_the_handle_entry_point_on_two_calls_in_a_row():
     B.hdet_converge_static(first.descriptors(), 8, 0, stream)
     torch.cuda.synchronize()
     assert torch.equal(first.param, want_first)
+    # what the entry point is for: further calls leave the device's free memory exactly as it was
+    # (the first call above already loaded the module and resolved the array's address)
+    free_before = torch.cuda.mem_get_info()[0]
+    B.hdet_converge_static(first.descriptors(), 8, 0, stream)
+    B.hdet_converge_static(second.descriptors(), 3, 0, stream)
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free_before
+    # a capturing stream is refused (the tables come from host memory that does not outlive the call),
+    # and the refusal leaves the capture usable
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        with pytest.raises(B.HdetError) as e:
+            B.hdet_converge_static(second.descriptors(), 3, 0, torch.cuda.current_stream().cuda_stream)
+        assert e.value.status == B.HDET_ERR_UNSUPPORTED and "captured" in e.value.message
+        second.param.add_(0.0)                  # something for the graph to hold
+    torch.cuda.synchronize()
