@@ -1,6 +1,6 @@
 """Benchmark of the HDET hot path on B200: fan-out update + converge + controller call, one step per launch.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload config4] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload config4] [--impl ours|reference] [--shard-replicas]
 
 A step is one pass of the whole hot path over the resident workload: hdet_step (spread and schedule
 scalars on the host, one fused fan-out update kernel; on the last update of a round the same kernel also
@@ -10,6 +10,8 @@ update+converge kernel, 147 GB resident); it falls back to the 350 M list when t
 free memory.  Gradients are generated once on the device and held fixed during timing (147 GB of
 inputs is far larger than L2, so no flush is needed).  With --gpus N > 1 every rank runs an
 independent copy of the workload on its own GPU (the path has no inter-GPU exchange): weak scaling.
+--shard-replicas instead splits the N replicas over the ranks, with an all-reduce of the local sums at
+every round end (strong scaling).  --gpus N > 1 without a launcher starts the N ranks itself.
 
 Prints ONE JSON line on rank 0.
 """
@@ -64,7 +66,7 @@ def measured_peaks():
     return FALLBACK_HBM_GBS, "fallback (6.65 TB/s, earlier measurement on this pool)"
 
 
-def oracle_sample(w: W.Workload, n_slabs: int = 32, slab: int = 65536):
+def oracle_sample(w: W.Workload, n_slabs: int, slab: int = 65536):
     """Bounded sample of the workload for the CPU oracle: n_slabs ranges of `slab` elements from the largest tensors."""
     big = sorted(range(len(w.tensors)), key=lambda k: -w.tensors[k].numel)
     slabs = []
@@ -77,33 +79,45 @@ def oracle_sample(w: W.Workload, n_slabs: int = 32, slab: int = 65536):
 
 
 class OracleBench:
-    """The CPU oracle, as it stands, on a bounded sample (numpy, one thread)."""
+    """The CPU oracle, as it stands, on a bounded sample, one worker process per usable host core.
 
-    def __init__(self, w: W.Workload):
-        sys.path.insert(0, os.path.join(ROOT, "tests"))
-        import harness as H
+    Every worker holds its own share of the sample (8 ranges of 65,536 elements x N replicas) and runs the
+    oracle's step on it with the gradients held fixed, as on the GPU; all workers run at the same time and the
+    wall time of the slowest counts.  The worker processes are started with `spawn` (a process forked after the
+    first CUDA call would hang).
+    """
+    SLABS_PER_WORKER = 8
+
+    def __init__(self, w: W.Workload, cores=None):
+        from oracle import driver as OD                      # test infrastructure: only this leg may use it
         self.w = w
-        self.slabs = oracle_sample(w)
-        self.run = H.OracleRun(w, self.slabs)
-        self.grads = self.run.grads(0)                      # held fixed, as on the GPU
+        self.cores = cores or OD.usable_cores()
+        self.slabs = oracle_sample(w, self.SLABS_PER_WORKER * self.cores)
+        self.pool = OD.OraclePool(w, self.slabs, n_workers=self.cores)
+        self.cores = self.pool.n_workers
         self.units = sum(n for (_, _, n) in self.slabs) * w.n_replicas
 
-    def step(self):
-        self.run.o.step(self.grads, R.step_losses(self.w, self.run.o.i % self.w.total_steps, self.run.o.perm_lr[0]))
+    def time_steps(self, steps: int) -> float:
+        return self.pool.time_steps(steps)
+
+    def close(self):
+        self.pool.close()
 
     def describe(self):
         return (f"{len(self.slabs)} ranges x {self.slabs[0][2]} elements x N={self.w.n_replicas} replicas of "
-                f"{self.w.name} ({self.units} replica-elements per step), gradients held fixed")
+                f"{self.w.name} ({self.units} replica-elements per step) split over {self.cores} worker processes, "
+                f"gradients held fixed")
 
 
-def time_oracle(w, steps, warmup):
-    ob = OracleBench(w)
-    for _ in range(warmup):
-        ob.step()
-    t0 = time.perf_counter()
-    for _ in range(steps):
-        ob.step()
-    dt = time.perf_counter() - t0
+def time_oracle(w, steps, warmup, cores=None):
+    """(bench object, replica-elements per second over all workers, seconds per step)."""
+    ob = OracleBench(w, cores)
+    try:
+        if warmup:
+            ob.time_steps(warmup)
+        dt = ob.time_steps(steps)
+    finally:
+        ob.close()
     return ob, ob.units * steps / dt, dt / steps
 
 
@@ -412,12 +426,175 @@ def run_ours(args):
         "device_status": int(final_state.device_status),
     }
     if world == 1 and not args.no_cpu_baseline:
-        ob, v, sec = time_oracle(w, args.cpu_steps, 1)
-        out["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": ob.describe(),
-                               "s_per_step": sec, "steps": args.cpu_steps}
+        ob, v, sec = time_oracle(w, args.cpu_steps, 1, args.cpu_cores)
+        out["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": ob.cores, "host_cpu_count": os.cpu_count(),
+                               "kind": "oracle", "sample": ob.describe(), "s_per_step": sec, "steps": args.cpu_steps}
     print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()
+
+
+def gather_round_losses(local_means, world: int, device="cpu"):
+    """Algorithm 1's all-gather of the per-replica round losses: every rank contributes the means of its local
+    replicas and receives all N, in replica order (ranks hold consecutive replicas)."""
+    if world == 1:
+        return [float(x) for x in local_means]
+    import torch
+    import torch.distributed as dist
+    mine = torch.tensor(list(local_means), dtype=torch.float64, device=device)
+    parts = [torch.empty_like(mine) for _ in range(world)]
+    dist.all_gather(parts, mine)
+    return [float(x) for p in parts for x in p.cpu()]
+
+
+def local_replica_range(n_replicas: int, world: int, rank: int):
+    """Replicas [first, first + count) held by `rank` when N replicas are split evenly over `world` ranks."""
+    if n_replicas % world:
+        raise SystemExit(f"--shard-replicas needs the replica count {n_replicas} to be a multiple of the {world} ranks")
+    count = n_replicas // world
+    return rank * count, count
+
+
+def run_sharded(args):
+    """Replica axis sharded over the ranks (the paper's own arrangement): every rank holds N / world replicas.
+
+    Per step hdet_step_sharded; at a round end the fused kernel leaves the sums over the local replicas in a
+    staging buffer, the ranks all-reduce it (the one exchange of Eq. 3, P floats), hdet_apply_mean writes
+    sum / N to the local replicas, the round losses are all-gathered (N doubles) and hdet_autolr_update runs
+    the controller on every rank.  Total work is fixed as ranks are added: strong scaling.
+    """
+    import torch
+    import torch.distributed as dist
+
+    from hdet_inputs import device as D
+    from paper_2604_24708_b200 import binding as B
+    from paper_2604_24708_b200 import from_workload
+    from paper_2604_24708_b200.arena import StackedArena
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+    w, note = pick_workload(args.workload, torch, args.sync_interval)
+    n, P = w.n_replicas, w.numel
+    first, n_local = local_replica_range(n, world, rank)
+    arena = StackedArena([t.numel for t in w.tensors], [t.group for t in w.tensors], n_local, w.optimizer, w.grad_dtype,
+                         device=dev, align_elems=w.align_elems)
+    D.fill(arena.param[0], R.param_key(w), 0, R.param_scale(w))
+    for r in range(1, n_local):
+        arena.param[r].copy_(arena.param[0])
+    for r in range(n_local):                                  # local replica r is global replica first + r
+        D.fill(arena.grad[r], R.grad_key(w, 0, first + r), 0, R.grad_scale(w))
+    h = B.hdet_create(from_workload.config_for(w, fuse=1, device=local, n_local=n_local, replica_offset=first),
+                      arena.descriptors())
+    B.hdet_set_schedule(h, from_workload.schedule_for(w))
+    _, total = B.hdet_partial_layout(h, len(w.tensors))
+    partial = torch.zeros(total, dtype=torch.float32, device=dev)
+    stream = torch.cuda.current_stream()
+    acc = [0.0] * n_local
+    state = {"i": 0, "n_acc": 0, "rounds": 0}
+    ar_events = []
+
+    def one_step(timed=False):
+        i = state["i"]
+        perm0 = list(B.hdet_get_state(h).perm_lr[0])[:n]
+        losses = R.step_losses(w, i % w.total_steps, perm0)
+        for r in range(n_local):
+            acc[r] += float(losses[first + r])
+        state["n_acc"] += 1
+        if B.hdet_step_sharded(h, None, partial, stream.cuda_stream):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            if world > 1:
+                dist.all_reduce(partial)                       # on the current (= launch) stream's order
+            b.record(stream)
+            if timed:
+                ar_events.append((a, b))
+            B.hdet_apply_mean(h, partial, stream.cuda_stream)
+            means = [x / state["n_acc"] for x in acc]
+            B.hdet_autolr_update(h, gather_round_losses(means, world, dev))
+            for r in range(n_local):
+                acc[r] = 0.0
+            state["n_acc"] = 0
+            state["rounds"] += 1
+        state["i"] += 1
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        one_step()
+    barrier()
+    sampler = ClockSampler(local) if rank == 0 else None
+    launches0 = B.hdet_kernel_launches(h)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record(stream)
+    for _ in range(args.steps):
+        one_step(timed=True)
+    e1.record(stream)
+    barrier()
+    clocks = sampler.stop() if sampler else None
+    launches = B.hdet_kernel_launches(h) - launches0
+    ms_per_step = max_over_ranks(e0.elapsed_time(e1), world, dev) / args.steps
+    ar_ms = sum(a.elapsed_time(b) for a, b in ar_events)
+    ar_ms = max_over_ranks(ar_ms, world, dev)
+    final_state = B.hdet_get_state(h, raise_on_nonfinite=False)
+    B.hdet_destroy(h)
+    if rank == 0:
+        value = n * P / (ms_per_step * 1e-3)                   # all N replicas of the one job, whatever the rank count
+        bpe = bytes_per_element(w)
+        peak, peak_src = measured_peaks()
+        rounds = max(1, len(ar_events))
+        # per GPU and step: the local update (26 B per local replica-element); per round end additionally the
+        # staging buffer written (4 B per parameter), read and the mean written to the local replicas
+        local_bytes = bpe * n_local * P
+        achieved = local_bytes * world / (ms_per_step * 1e-3) / 1e9
+        out = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "strong",
+            "vs_baseline": None, "dtype": "f32 (bf16 gradients, fp64 replica sum)" if w.grad_dtype == W.DTYPE_BF16 else "f32",
+            "data": "synthetic (seeded integer generator; gradients held fixed during timing)",
+            "config": {"workload": w.name, "n_replicas": n, "replicas_per_gpu": n_local, "params_per_replica": P,
+                       "sync_interval": w.sync_interval, "l2_policy": "inputs larger than L2 (no flush)",
+                       "parallelism": f"replica axis sharded over {world} GPU(s): hdet_step_sharded, all-reduce of "
+                                      f"{total} fp32 sums per round, hdet_apply_mean", "note": note},
+            "gpu_launches": int(launches), "clocks": clocks,
+            "allreduce": {"rounds_timed": len(ar_events), "ms_per_round": ar_ms / rounds,
+                          "share_of_step_time": ar_ms / (ms_per_step * args.steps), "bytes_per_round": 4 * total},
+            "roofline": {"bound": "hbm", "achieved": achieved / world, "peak": peak, "unit": "GB/s",
+                         "frac": achieved / world / peak, "traffic": None, "peak_source": peak_src,
+                         "kernel": "fanout_kernel (per GPU; algorithmic bytes of the update only)",
+                         "bytes_per_element": bpe},
+            "e2e": None, "device_status": int(final_state.device_status),
+        }
+        print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def relaunch_under_torchrun(args):
+    """`--gpus N` without a launcher: start the N ranks here (what the driver's torchrun line does)."""
+    import socket
+    if args.impl == "ours":
+        import torch
+        have = torch.cuda.device_count() if torch.cuda.is_available() else 0
+        if have < args.gpus:
+            raise SystemExit(f"bench.py --gpus {args.gpus}: only {have} CUDA device(s) visible; "
+                             f"nothing was run (a smaller run would misreport n_gpus)")
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    raise SystemExit(subprocess.run(cmd).returncode)
 
 
 def run_reference(args):
@@ -425,7 +602,7 @@ def run_reference(args):
     if int(os.environ.get("RANK", "0")) != 0:
         return
     w = W.ALL_CONFIGS[args.workload]()
-    ob, v, sec = time_oracle(w, args.steps, max(args.warmup, 1))
+    ob, v, sec = time_oracle(w, args.steps, max(args.warmup, 1), args.cpu_cores)
     world = int(os.environ.get("WORLD_SIZE", "1"))
     out = {
         "impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -433,7 +610,8 @@ def run_reference(args):
         "vs_baseline": None, "dtype": "f64", "data": "synthetic (seeded integer generator)",
         "config": {"workload": w.name, "n_replicas": w.n_replicas, "params_per_replica": w.numel,
                    "sample": ob.describe()},
-        "cpu_baseline": {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": ob.describe()},
+        "cpu_baseline": {"value": v, "unit": UNIT, "cores": ob.cores, "host_cpu_count": os.cpu_count(), "kind": "oracle",
+                         "sample": ob.describe()},
         "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -459,13 +637,25 @@ def main():
                     help="one pair of Adam moments for all replicas (needs --shared-grad or --grad-mode mean)")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-steps", type=int, default=30)
+    ap.add_argument("--cpu-cores", type=int, default=None,
+                    help="worker processes of the CPU oracle (default: every core this process may use)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-per-kernel", action="store_true", help="skip the per-kernel timings that follow the headline run")
     ap.add_argument("--traffic-bytes", type=float, default=None,
                     help="dram bytes per launch of the dominant kernel from an ncu capture (reported as roofline.traffic)")
+    ap.add_argument("--shard-replicas", action="store_true",
+                    help="split the replica axis over the ranks (N / world replicas per GPU, all-reduce of the local "
+                         "sums at every round end) instead of running one independent copy of the job per GPU")
     args = ap.parse_args()
+    world_env = os.environ.get("WORLD_SIZE")
+    if world_env is None and args.gpus > 1:
+        relaunch_under_torchrun(args)
+    if world_env is not None and int(world_env) != args.gpus:
+        raise SystemExit(f"bench.py: --gpus {args.gpus} disagrees with WORLD_SIZE={world_env} set by the launcher")
     if args.impl == "reference":
         run_reference(args)
+    elif args.shard_replicas:
+        run_sharded(args)
     else:
         run_ours(args)
 

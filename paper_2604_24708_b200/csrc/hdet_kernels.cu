@@ -307,8 +307,8 @@ __device__ __forceinline__ void tile_vector(const TensorDesc& td, long long off,
 // pipeline below this takes the address arithmetic and the load/store instructions of 26 bytes per
 // element off the consumer warps and keeps more bytes in flight per SM; the arithmetic per element, and
 // so every result bit, is the same.
-// With the gradient replica-mean the ring first carries the N gradient tiles alone (the consumers form
-// g_bar in fp64, r = 0..N-1), then the N (theta, m, v) stages.
+// With the gradient replica-mean the ring first carries the gradient tiles alone, several replicas per
+// stage (the consumers form g_bar in fp64, r = 0..N-1), then the N (theta, m, v) stages.
 constexpr int kProducerThreads = 32;
 constexpr int kStages = 3;
 constexpr int kMaxDevices = 64;
@@ -347,7 +347,11 @@ __device__ __forceinline__ void tile_bulk(const TensorDesc& td, long long off, c
                                           const AdamConsts& c, bool& bad, unsigned char* smem, unsigned* status) {
   using L = BulkLayout<GradT>;
   const int n = s.n_replicas;
-  const int n_items = kMean ? 2 * n : n;      // with the gradient mean: N gradient-only items, then N replicas
+  // With the gradient mean the ring first carries the gradient tiles alone, as many replicas per stage as fit
+  // (7 for bf16, 4 for fp32), then the N replicas.
+  constexpr int kGradPerItem = L::kStageBytes / L::kGradBytes;
+  const int n_grad_items = kMean ? (n + kGradPerItem - 1) / kGradPerItem : 0;
+  const int n_items = n_grad_items + n;
   const uint32_t base = bulk::smem_addr(smem);
   const uint32_t full = base + L::kBarrierOff, done = full + 8 * kStages, mean_done = done + 8 * kStages;
   float* const P = td.param + off;
@@ -362,12 +366,13 @@ __device__ __forceinline__ void tile_bulk(const TensorDesc& td, long long off, c
     auto request = [&](int i) {
       const int st = i % kStages;
       const uint32_t slot = base + st * L::kStageBytes, bar = full + 8 * st;
-      if (kMean && i < n) {
-        bulk::barrier_expect(bar, L::kGradBytes);
-        bulk::load(slot + 3 * L::kF32Bytes, G + i * gs, L::kGradBytes, bar);
+      if (i < n_grad_items) {
+        const int r0 = i * kGradPerItem, count = n - r0 < kGradPerItem ? n - r0 : kGradPerItem;
+        bulk::barrier_expect(bar, count * L::kGradBytes);
+        for (int q = 0; q < count; ++q) bulk::load(slot + q * L::kGradBytes, G + (r0 + q) * gs, L::kGradBytes, bar);
         return;
       }
-      const int r = kMean ? i - n : i;
+      const int r = i - n_grad_items;
       bulk::barrier_expect(bar, kMean ? 3 * L::kF32Bytes : L::kStageBytes);
       bulk::load(slot, P + r * ps, L::kF32Bytes, bar);
       bulk::load(slot + L::kF32Bytes, M + r * ss, L::kF32Bytes, bar);
@@ -379,8 +384,8 @@ __device__ __forceinline__ void tile_bulk(const TensorDesc& td, long long off, c
     for (int i = 0; i < n_items; ++i) {
       const int st = i % kStages;
       if (!bulk::barrier_wait(done + 8 * st, (i / kStages) & 1)) { alive = false; break; }
-      if (!(kMean && i < n)) {
-        const int r = kMean ? i - n : i;
+      if (i >= n_grad_items) {
+        const int r = i - n_grad_items;
         const uint32_t slot = base + st * L::kStageBytes;
         if (!kConv) bulk::store(P + r * ps, slot, L::kF32Bytes);
         bulk::store(M + r * ss, slot + L::kF32Bytes, L::kF32Bytes);
@@ -425,16 +430,19 @@ __device__ __forceinline__ void tile_bulk(const TensorDesc& td, long long off, c
     for (int k = 0; k < kTileVecs; ++k)
 #pragma unroll
       for (int q = 0; q < 4; ++q) acc[k][q] = 0.0;
-    for (; i < n; ++i) {
+    for (; i < n_grad_items; ++i) {
       const int st = i % kStages;
       if (!bulk::barrier_wait(full + 8 * st, (i / kStages) & 1)) { atomicOr(status, 2u); return; }
-      const unsigned char* slot = smem + st * L::kStageBytes + 3 * L::kF32Bytes;
+      const int r0 = i * kGradPerItem, count = n - r0 < kGradPerItem ? n - r0 : kGradPerItem;
+      for (int r = 0; r < count; ++r) {        // replicas in order, so the sum is the one of the register path
+        const unsigned char* slot = smem + st * L::kStageBytes + r * L::kGradBytes;
 #pragma unroll
-      for (int k = 0; k < kTileVecs; ++k) {
-        float g[4];
-        read_grad(slot, k * kThreads + threadIdx.x, g, GradT{});
+        for (int k = 0; k < kTileVecs; ++k) {
+          float g[4];
+          read_grad(slot, k * kThreads + threadIdx.x, g, GradT{});
 #pragma unroll
-        for (int q = 0; q < 4; ++q) acc[k][q] += (double)g[q];
+          for (int q = 0; q < 4; ++q) acc[k][q] += (double)g[q];
+        }
       }
       bulk::barrier_arrive(done + 8 * st);
     }
@@ -452,7 +460,7 @@ __device__ __forceinline__ void tile_bulk(const TensorDesc& td, long long off, c
       for (int q = 0; q < 4; ++q) sum[k][q] = 0.0;
   }
   for (; i < n_items; ++i) {
-    const int r = kMean ? i - n : i;
+    const int r = i - n_grad_items;
     const int st = i % kStages;
     if (!bulk::barrier_wait(full + 8 * st, (i / kStages) & 1)) { atomicOr(status, 2u); return; }
     unsigned char* const slot = smem + st * L::kStageBytes;

@@ -8,6 +8,9 @@ import numpy as np
 from hdet_inputs import recipes as R
 from hdet_inputs import workloads as W
 from oracle import hdet_oracle as O
+# The oracle's driver (slab selection, seeded inputs, worker processes, error measure) lives beside the oracle.
+from oracle.driver import (OraclePool, OracleRun, Slab, edge_slabs, oracle_for, random_run_slabs,  # noqa: F401
+                           rel_err, slab_elements, whole_tensor_slabs)
 
 
 # ----------------------------------------------------------------------------- library side
@@ -93,86 +96,7 @@ class GpuRun:
         self.torch.cuda.empty_cache()
 
 
-# ----------------------------------------------------------------------------- oracle side
-Slab = Tuple[int, int, int]   # (tensor index, first element inside the tensor, length)
-
-
-def oracle_for(w: W.Workload, params: Sequence[np.ndarray], groups: Sequence[int],
-               grad_mean: bool = False) -> O.HdetOracle:
-    return O.HdetOracle(
-        params, groups, w.n_groups, optimizer=w.optimizer, total_steps=w.total_steps, sched_kind=w.sched_kind,
-        max_lr=list(w.max_lr), weight_decay=list(w.weight_decay), pct_start=w.pct_start, div_factor=w.div_factor,
-        final_div_factor=w.final_div_factor, alpha_lr=w.alpha_lr, alpha_wd=w.alpha_wd,
-        sync_interval=w.sync_interval, autolr=bool(w.autolr), warmup_steps=w.warmup_steps, ctrl_beta=w.ctrl_beta,
-        ctrl_sigma=w.ctrl_sigma, ctrl_lambda=w.ctrl_lambda, f_div=w.f_div, f_final=w.f_final,
-        reshuffle=bool(w.reshuffle), seed=w.seed, beta1=w.beta1, beta2=w.beta2, eps=w.eps, n_replicas=w.n_replicas,
-        grad_mean=grad_mean, momentum=w.momentum, auto_wd=bool(w.auto_wd))
-
-
-class OracleRun:
-    """The oracle over chosen element ranges (slabs) of the workload, with the same seeded inputs."""
-
-    def __init__(self, w: W.Workload, slabs: Sequence[Slab], shared_grad: bool = False, grad_mean: bool = False,
-                 loss_dtype: str = "float64"):
-        self.w, self.slabs, self.shared_grad = w, list(slabs), shared_grad
-        self.loss_dtype = loss_dtype
-        offs = w.arena_offsets()
-        self.starts = [offs[k] + s for (k, s, n) in self.slabs]
-        params = [np.tile(R.param_slab(w, a, n).astype(np.float64), (w.n_replicas, 1))
-                  for a, (k, s, n) in zip(self.starts, self.slabs)]
-        self.o = oracle_for(w, params, [w.tensors[k].group for (k, s, n) in self.slabs], grad_mean=grad_mean)
-        self.i = 0
-
-    def grads(self, step: int) -> List[np.ndarray]:
-        w = self.w
-        out = []
-        for a, (k, s, n) in zip(self.starts, self.slabs):
-            if self.shared_grad:
-                out.append(R.grad_slab(w, step, 0, a, n).astype(np.float64))
-            else:
-                out.append(np.stack([R.grad_slab(w, step, r, a, n) for r in range(w.n_replicas)]).astype(np.float64))
-        return out
-
-    def step(self) -> bool:
-        losses = R.step_losses(self.w, self.i, self.o.perm_lr[0])
-        if self.loss_dtype == "float32":           # what the library reads from an fp32 loss tensor, exactly
-            losses = losses.astype(np.float32).astype(np.float64)
-        ended = self.o.step(self.grads(self.i), losses)
-        self.i += 1
-        return ended
-
-
-def whole_tensor_slabs(w: W.Workload) -> List[Slab]:
-    return [(k, 0, t.numel) for k, t in enumerate(w.tensors)]
-
-
-def sampled_slabs(w: W.Workload, tile: int = 2048, extra: int = 2, seed: int = 0) -> List[Slab]:
-    """First and last tile of every tensor (tails included) plus `extra` random tiles of each large tensor."""
-    rng = np.random.default_rng(seed)
-    out: List[Slab] = []
-    for k, t in enumerate(w.tensors):
-        n = t.numel
-        if n <= 2 * tile:
-            out.append((k, 0, n))
-            continue
-        out.append((k, 0, tile))
-        last = max(tile, (n - 1) // tile * tile - tile)      # the last full tile together with the ragged tail
-        out.append((k, last, n - last))
-        n_tiles = n // tile
-        for j in rng.choice(np.arange(1, max(2, n_tiles - 1)), size=min(extra, max(0, n_tiles - 2)), replace=False):
-            out.append((k, int(j) * tile, tile))
-    return out
-
-
 # ----------------------------------------------------------------------------- comparison
-def rel_err(got: np.ndarray, ref: np.ndarray) -> np.ndarray:
-    """|got - ref| / max(|ref|, RMS(ref)): per-element relative error with an RMS floor near zero."""
-    ref = np.asarray(ref, dtype=np.float64)
-    rms = float(np.sqrt(np.mean(ref * ref)))
-    den = np.maximum(np.abs(ref), rms if rms > 0 else 1.0)
-    return np.abs(np.asarray(got, dtype=np.float64) - ref) / den
-
-
 def compare_slabs(g: GpuRun, o: OracleRun, tol: float, check_moments: bool = True) -> float:
     """Largest relative error over all slabs (params and, for AdamW, both moments); asserts it is <= tol."""
     worst = 0.0

@@ -35,7 +35,10 @@ def test_bench_line_has_the_contract_keys():
     e = d["e2e"]
     assert e["h2d_bytes_per_step"] == 8 * 25_190_400 * 2 and e["d2h_bytes_per_step"] > 0 and 0 < e["value"] < d["value"]
     c = d["cpu_baseline"]
-    assert c["kind"] == "oracle" and c["cores"] == 1 and c["value"] > 0 and c["unit"] == d["unit"]
+    assert c["kind"] == "oracle" and c["value"] > 0 and c["unit"] == d["unit"]
+    assert 1 <= c["cores"] <= c["host_cpu_count"] and f"{c['cores']} worker processes" in c["sample"]
+    if c["host_cpu_count"] > 1 and len(os.sched_getaffinity(0)) > 1:
+        assert c["cores"] > 1                                       # the oracle is timed on all usable host cores
     assert set(d["clocks"]) >= {"sm_mhz", "sm_max_mhz", "reasons"}
     assert d["device_status"] == 0
 
@@ -46,3 +49,13 @@ def test_bench_device_stepping_and_shared_moments_modes_run():
     assert d["config"]["stepping"] == "device" and d["gpu_launches"] == 8    # scalar kernel + fan-out per step
     d = _run("--shared-grad", "--shared-state", "--no-cpu-baseline", "--no-per-kernel")
     assert d["roofline"]["bytes_per_element"] == pytest.approx(10.25)
+
+
+@pytest.mark.gpu
+def test_bench_sharded_replica_mode_runs_on_one_rank():
+    """--shard-replicas with one rank: hdet_step_sharded + hdet_apply_mean (no all-reduce partner), strong-scaling units."""
+    d = _run("--shard-replicas", "--sync-interval", "2", "--no-cpu-baseline")
+    assert d["scaling"] == "strong" and d["n_gpus"] == 1 and d["config"]["replicas_per_gpu"] == 8
+    assert d["gpu_launches"] == 4 + 2                                # four updates, two of them followed by hdet_apply_mean
+    assert d["allreduce"]["rounds_timed"] == 2 and d["device_status"] == 0
+    assert d["value"] == pytest.approx(8 * 25_190_400 / (d["ms_per_step"] * 1e-3), rel=1e-6)

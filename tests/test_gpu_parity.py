@@ -366,21 +366,6 @@ def test_config2_full_run_sampled():
     assert worst <= TOL_FULL_RUN
 
 
-def _decoder_sample(w, n_small=12, n_big=10, seed=0):
-    """First tile of some small tensors; first, last (ragged tail) and a random tile of some matrices."""
-    rng = np.random.default_rng(seed)
-    small = [k for k, t in enumerate(w.tensors) if t.numel <= 8192]
-    big = [k for k, t in enumerate(w.tensors) if t.numel > 8192]
-    slabs = [(int(k), 0, w.tensors[k].numel if w.tensors[k].numel <= 2048 else 2048)
-             for k in rng.choice(small, n_small, replace=False)]
-    picks = [0, 1, big[-1]] + [int(k) for k in rng.choice(big[2:-1], n_big - 3, replace=False)]
-    for k in picks:
-        n = w.tensors[k].numel
-        j = int(rng.integers(1, n // 2048 - 1))
-        slabs += [(k, 0, 2048), (k, n - 2048 - 1000, 2048 + 1000), (k, j * 2048, 2048)]
-    return slabs
-
-
 def _free_gb():
     import gc
     import torch
@@ -389,12 +374,72 @@ def _free_gb():
     return torch.cuda.mem_get_info()[0] / 1e9
 
 
+ONE_STEP_FRACTION = 0.05
+
+
+def _full_size(w, check_every):
+    """A full-size workload against the oracle, with the coverage stated and asserted.
+
+    Whole run, every update: the first tile and the last tile with its ragged tail of EVERY tensor (oracle
+    worker processes in lockstep with the GPU; checked after the first update, every `check_every` updates and
+    at the end, scalars at every round end).  After the first update, at the one-step tolerance, also at least
+    5 % of all elements in random runs of 64 tiles (each run is an independent one-step oracle problem, farmed
+    out to a process pool).  Returns the worst relative error seen.
+    """
+    import multiprocessing as mp
+    from oracle import driver as OD
+    edge = H.edge_slabs(w)
+    assert {k for (k, _, _) in edge} == set(range(len(w.tensors)))            # every tensor is touched
+    runs = H.random_run_slabs(w, ONE_STEP_FRACTION, run_tiles=64, seed=w.seed)
+    one_step_fraction = H.slab_elements(runs) / w.numel
+    whole_run_fraction = H.slab_elements(edge) / w.numel
+    assert one_step_fraction >= ONE_STEP_FRACTION
+    pool = H.OraclePool(w, edge)
+    g = H.GpuRun(w)
+    names = ("param", "m", "v")
+
+    def fetch(k, s, n):
+        return {name: g.slab(name, k, s, n) for name in names}
+
+    worst, o_perm = 0.0, list(range(w.n_replicas))
+    try:
+        for i in range(w.total_steps):
+            perm = g.perm0()
+            assert perm == o_perm
+            ended = g.step(perm)
+            o_ended, o_perm = pool.step()
+            assert ended == o_ended
+            if i == 0:
+                worst = max(worst, pool.compare(fetch, TOL_ONE_STEP))
+                groups = [runs[j:j + 4] for j in range(0, len(runs), 4)]
+                tasks = ((w, grp, [fetch(*sl) for sl in grp], TOL_ONE_STEP, {}) for grp in groups)
+                with mp.get_context("spawn").Pool(OD.usable_cores()) as farm:
+                    for e, msg in farm.imap_unordered(OD.one_step_errors, tasks):
+                        assert msg is None, msg
+                        worst = max(worst, e)
+            elif (i + 1) % check_every == 0:
+                worst = max(worst, pool.compare(fetch, TOL_FULL_RUN))
+            if ended or i == 0:
+                H.compare_scalars(g.state(), pool.scalars(), w.n_replicas, w.n_groups)
+        worst = max(worst, pool.compare(fetch, TOL_FULL_RUN))
+        st = g.state()
+        assert st.device_status == 0
+        H.compare_scalars(st, pool.scalars(), w.n_replicas, w.n_groups)
+    finally:
+        pool.close()
+        g.close()
+    print(f"\n{w.name}: checked {100 * one_step_fraction:.2f} % of the N x P = {w.n_replicas} x {w.numel} elements after one "
+          f"update and {100 * whole_run_fraction:.3f} % through all {w.total_steps} updates (first and last tile of each of "
+          f"the {len(w.tensors)} tensors, all touched); worst relative error {worst:.2e}")
+    return worst
+
+
 def test_config3_full_size_sampled():
     """N=8, 354.8 M parameters in 292 tensors (39.7 GB resident), 500 updates, T=100, controller on."""
     w = W.config3()
     if _free_gb() < 45:
         pytest.skip("needs 45 GB of free device memory")
-    _lockstep(w, _decoder_sample(w, 10, 8), check_every=250)
+    assert _full_size(w, check_every=250) <= TOL_FULL_RUN
 
 
 def test_config4_full_size_sampled():
@@ -402,7 +447,7 @@ def test_config4_full_size_sampled():
     w = W.config4()
     if _free_gb() < 152:
         pytest.skip("needs 152 GB of free device memory")
-    _lockstep(w, _decoder_sample(w, 12, 10), check_every=10)
+    assert _full_size(w, check_every=10) <= TOL_FULL_RUN
 
 
 @pytest.mark.parametrize("T", [1, 10, 100])
@@ -411,7 +456,7 @@ def test_config5_n16_weight_decay_spread(T):
     w = W.config5(T)
     if _free_gb() < 32:
         pytest.skip("needs 32 GB of free device memory")
-    _lockstep(w, _decoder_sample(w, 6, 5), check_every=100)
+    assert _full_size(w, check_every=100) <= TOL_FULL_RUN
 
 
 @pytest.mark.parametrize("align", [8, 1])
