@@ -206,6 +206,26 @@ def converge(theta: np.ndarray) -> None:
         theta[r] = mean
 
 
+def bf16_bits(x: np.ndarray) -> np.ndarray:
+    """The bfloat16 image of single-precision values, as 16-bit patterns, rounding to nearest, ties to even.
+
+    Section 3.3's averaged parameters (Eq. 3) are what the next forward pass of Algorithm 1 reads; a
+    mixed-precision model reads them as bfloat16.  The paper does not say how that copy is made.  Reading
+    taken: it is the stored single-precision parameter rounded once to bfloat16, which keeps the upper 16 bits
+    of the fp32 pattern: add 0x7FFF plus the lowest kept bit to the pattern, then drop the lower 16 bits.
+    (Finite inputs only; the path never stores a NaN here without flagging it.)
+    """
+    u = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32).astype(np.uint64)
+    keep_lsb = (u >> np.uint64(16)) & np.uint64(1)
+    return ((u + np.uint64(0x7FFF) + keep_lsb) >> np.uint64(16)).astype(np.uint16)
+
+
+def averaged_bf16(theta: np.ndarray) -> np.ndarray:
+    """bfloat16 copy of the averaged parameters after Eq. 3: replica 0 of `theta` ([N, numel], double, all rows
+    equal after converge) rounded to single precision (the stored master value), then to bfloat16."""
+    return bf16_bits(theta[0].astype(np.float32))
+
+
 # --------------------------------------------------------------------------- #
 # Algorithm 1
 # --------------------------------------------------------------------------- #

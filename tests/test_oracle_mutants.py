@@ -101,6 +101,12 @@ MUTANTS = [
     ("if self.grad_mean and gk.ndim == 2:", "if False:"),
     ("self.v[k][r], g_r, lr[g_id][r], wd[g_id][r],", "self.v[k][r], g_r, lr[g_id][r], self.weight_decay[g_id],"),
     ("g_r, lr[g_id][r], wd[g_id][r], self.momentum)", "g_r, lr[g_id][r], self.weight_decay[g_id], self.momentum)"),
+    # bfloat16 copy of the averaged parameters
+    ("return ((u + np.uint64(0x7FFF) + keep_lsb) >> np.uint64(16)).astype(np.uint16)",
+     "return (u >> np.uint64(16)).astype(np.uint16)"),
+    ("return ((u + np.uint64(0x7FFF) + keep_lsb) >> np.uint64(16)).astype(np.uint16)",
+     "return ((u + np.uint64(0x8000)) >> np.uint64(16)).astype(np.uint16)"),
+    ("return bf16_bits(theta[0].astype(np.float32))", "return bf16_bits(theta[0].astype(np.float32) * 2)"),
 ]
 
 

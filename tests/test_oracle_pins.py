@@ -667,3 +667,41 @@ def test_remark1_weight_decay_channel_controller():
     # the tables of the next update use the new base
     _, _, wd = one.tables()
     assert wd[0].mean() == pytest.approx(one.wd_base[0], rel=1e-14)
+
+
+# --------------------------------------------------------------------------- bfloat16 copy of the averaged parameters
+def test_bf16_rounding_known_patterns_ties_and_the_library_conversion():
+    """Round to nearest, ties to even, on the fp32 bit pattern: textbook cases, the error bound, idempotence,
+    and agreement with the library's own fp32 -> bf16 conversion on random and on tie values."""
+    import torch
+
+    def f32(bits):
+        return np.array(bits, dtype=np.uint32).view(np.float32)
+
+    cases = {0x3F800000: 0x3F80,      # 1.0
+             0xBF800000: 0xBF80,      # -1.0
+             0x3F808000: 0x3F80,      # exactly half way above an even pattern: stays
+             0x3F818000: 0x3F82,      # half way above an odd pattern: goes up to the even one
+             0x3F808001: 0x3F81,      # just above half way: up
+             0x3F807FFF: 0x3F80,      # just below half way: down
+             0x00000000: 0x0000, 0x80000000: 0x8000,
+             0x477FE000: 0x4780}      # 65504.0: the carry runs into the exponent
+    got = O.bf16_bits(f32(list(cases)))
+    assert got.tolist() == list(cases.values())
+    rng = np.random.default_rng(5)
+    x = (rng.standard_normal(200000) * 10.0 ** rng.integers(-6, 6, 200000)).astype(np.float32)
+    ties = f32(((rng.integers(0, 0x7F7F, 4096, dtype=np.int64) << 16) | 0x8000).astype(np.uint32))   # finite exact ties
+    for v in (x, ties):
+        want = torch.from_numpy(v).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+        assert np.array_equal(O.bf16_bits(v), want)
+    back = (O.bf16_bits(x).astype(np.uint32) << 16).view(np.float32)
+    assert np.all(np.abs(back.astype(np.float64) - x) <= np.abs(x.astype(np.float64)) * 2.0 ** -8)   # half an ulp of 8 bits
+    assert np.array_equal(O.bf16_bits(back), O.bf16_bits(x))                                         # idempotent
+
+
+def test_averaged_bf16_is_the_rounded_master_copy_of_the_mean():
+    theta = np.array([[1.0, 3.0, 0.1], [2.0, 3.0, 0.3]])
+    O.converge(theta)
+    bits = O.averaged_bf16(theta)
+    assert bits.tolist() == O.bf16_bits(np.array([1.5, 3.0, 0.2], dtype=np.float32)).tolist()
+    assert bits[0] == 0x3FC0 and bits[1] == 0x4040
