@@ -19,6 +19,7 @@
  *   hdet_step_sharded / hdet_apply_mean / hdet_partial_layout   replica axis split over GPUs
  *   hdet_warm_init         warm noisy initialisation (Eq. 10)
  *   hdet_converge_static   allocation-free variant of hdet_converge
+ *   hdet_plan_tiles        host-only view of the work plan (tests, tools)
  *
  * Conventions
  *   - Every tensor pointer is a DEVICE pointer owned by the caller; it must stay
@@ -378,6 +379,22 @@ HDET_API int hdet_converge_static(const hdet_tensor* tensors, int64_t n_tensors,
 /* hdet_last_error -- text of the last failure on h (when h is NULL: of the last failed call
  * that has no handle, hdet_create or hdet_converge_static, on this thread).  The pointer stays valid until the next call on that handle. */
 HDET_API const char* hdet_last_error(hdet_handle h);
+
+/*
+ * hdet_plan_tiles -- (no counterpart in the paper: a host-only view of the work plan, for tests and tools.)
+ * Runs the checks of hdet_create on cfg and the descriptors and reports the plan hdet_create would build,
+ * without touching a device (the pointers are only inspected for alignment, never dereferenced):
+ *   *n_tiles              number of tiles; tile i covers elements [2048 * tile_index[i],
+ *                         min(numel, 2048 * (tile_index[i] + 1))) of tensor tile_tensor[i]
+ *   tile_tensor, tile_index   HOST arrays of `capacity` entries, or both NULL to query the count
+ *   tensor_access[k]      HOST, n_tensors entries or NULL: 0 = scalar accesses, 1 = 128-bit accesses,
+ *                         3 = 128-bit accesses and bulk copies of whole tiles (AdamW)
+ *   partial_offsets[k]    HOST, n_tensors entries or NULL: as hdet_partial_layout
+ * Errors: those of hdet_create's checks; INVALID_ARG when capacity is too small.
+ */
+HDET_API int hdet_plan_tiles(const hdet_config* cfg, const hdet_tensor* tensors, int64_t n_tensors, int32_t* tile_tensor,
+                             int32_t* tile_index, int64_t capacity, int64_t* n_tiles, int32_t* tensor_access,
+                             int64_t* partial_offsets);
 
 /* hdet_kernel_launches -- number of kernels this handle has launched so far. */
 HDET_API int64_t hdet_kernel_launches(hdet_handle h);

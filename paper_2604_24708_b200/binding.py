@@ -116,6 +116,10 @@ def _load() -> C.CDLL:
     lib.hdet_kernel_launches.restype = C.c_int64
     lib.hdet_converge_static.argtypes = [C.POINTER(hdet_tensor), C.c_int64, C.c_int32, C.c_int32, C.c_void_p]
     lib.hdet_converge_static.restype = C.c_int
+    lib.hdet_plan_tiles.argtypes = [C.POINTER(hdet_config), C.POINTER(hdet_tensor), C.c_int64, C.POINTER(C.c_int32),
+                                    C.POINTER(C.c_int32), C.c_int64, C.POINTER(C.c_int64), C.POINTER(C.c_int32),
+                                    C.POINTER(C.c_int64)]
+    lib.hdet_plan_tiles.restype = C.c_int
     for f in ("hdet_create", "hdet_set_schedule", "hdet_step", "hdet_converge", "hdet_autolr_update",
               "hdet_get_state", "hdet_set_state", "hdet_destroy"):
         getattr(lib, f).restype = C.c_int
@@ -243,6 +247,19 @@ def hdet_partial_layout(h, n_tensors: int):
     total = C.c_int64(0)
     _check(_lib.hdet_partial_layout(h, offs if n_tensors else None, n_tensors, C.byref(total)), h)
     return list(offs)[:n_tensors], int(total.value)
+
+
+def hdet_plan_tiles(cfg: hdet_config, tensors: Sequence[hdet_tensor]):
+    """The work plan hdet_create would build, computed on the host: (tile_tensor, tile_index, access per tensor,
+    partial-sum offset per tensor)."""
+    arr = (hdet_tensor * len(tensors))(*tensors) if tensors else None
+    count = C.c_int64(0)
+    _check(_lib.hdet_plan_tiles(C.byref(cfg), arr, len(tensors), None, None, 0, C.byref(count), None, None), None)
+    n = int(count.value)
+    tt, ti = (C.c_int32 * max(1, n))(), (C.c_int32 * max(1, n))()
+    acc, offs = (C.c_int32 * max(1, len(tensors)))(), (C.c_int64 * max(1, len(tensors)))()
+    _check(_lib.hdet_plan_tiles(C.byref(cfg), arr, len(tensors), tt, ti, n, C.byref(count), acc, offs), None)
+    return list(tt)[:n], list(ti)[:n], list(acc)[:len(tensors)], list(offs)[:len(tensors)]
 
 
 def hdet_warm_init(h, nu: float = 0.01, seed: int = 0, stream: int = 0) -> None:

@@ -198,17 +198,17 @@ DevConst device_constants(const hdet_ctx* h) {
   return c;
 }
 
-}  // namespace
+// What hdet_create derives from the descriptors before it touches a device: per-tensor device descriptors
+// (access path chosen from the alignment), the tile table and the layout of the partial-sum staging buffer.
+struct WorkPlan {
+  std::vector<TensorDesc> descs;
+  std::vector<Tile> tiles;
+  int64_t n_shared_state = 0;
+  int64_t partial_numel = 0;
+};
 
-namespace hdet {
-void set_handleless_error(const char* msg) { g_create_error = msg ? msg : ""; }
-}  // namespace hdet
-
-extern "C" {
-
-int hdet_create(const hdet_config* cfg, const hdet_tensor* tensors, int64_t n_tensors, hdet_handle* out) {
-  if (out) *out = nullptr;
-  if (!cfg || !out) return fail(nullptr, HDET_ERR_INVALID_ARG, "hdet_create: cfg and out must not be NULL");
+// Checks cfg and the descriptors and fills `out`.  Host arithmetic only.
+int plan_work(const hdet_config* cfg, const hdet_tensor* tensors, int64_t n_tensors, WorkPlan& out) {
   if (n_tensors < 0 || (n_tensors > 0 && !tensors))
     return fail(nullptr, HDET_ERR_INVALID_ARG, "hdet_create: tensors is NULL or n_tensors < 0");
   if (cfg->n_replicas < 1 || cfg->n_replicas > HDET_MAX_REPLICAS)
@@ -243,10 +243,10 @@ int hdet_create(const hdet_config* cfg, const hdet_tensor* tensors, int64_t n_te
     return fail(nullptr, HDET_ERR_UNSUPPORTED,
                 "hdet_create: with a sharded replica axis the gradient mean spans GPUs; all-reduce it and pass a shared gradient");
   const size_t gsz = cfg->grad_dtype == HDET_DTYPE_BF16 ? 2 : 4;
-  std::vector<TensorDesc> descs;
-  std::vector<Tile> tiles;
-  int64_t n_shared_state = 0;
-  int64_t partial_numel = 0;
+  std::vector<TensorDesc>& descs = out.descs;
+  std::vector<Tile>& tiles = out.tiles;
+  int64_t& n_shared_state = out.n_shared_state;
+  int64_t& partial_numel = out.partial_numel;
   const bool adamw = cfg->optimizer == HDET_OPT_ADAMW;
   const bool sgd_momentum = cfg->optimizer == HDET_OPT_SGD && cfg->momentum != 0.0;
   for (int64_t k = 0; k < n_tensors; ++k) {
@@ -306,6 +306,30 @@ int hdet_create(const hdet_config* cfg, const hdet_tensor* tensors, int64_t n_te
   if (n_shared_state != 0 && n_shared_state != n_tensors)
     return fail(nullptr, HDET_ERR_UNSUPPORTED, "hdet_create: state_stride 0 must be used by all tensors or by none");
 
+  return HDET_OK;
+}
+
+}  // namespace
+
+namespace hdet {
+void set_handleless_error(const char* msg) { g_create_error = msg ? msg : ""; }
+}  // namespace hdet
+
+extern "C" {
+
+int hdet_create(const hdet_config* cfg, const hdet_tensor* tensors, int64_t n_tensors, hdet_handle* out) {
+  TraceRange trace("hdet_create");
+  if (out) *out = nullptr;
+  if (!cfg || !out) return fail(nullptr, HDET_ERR_INVALID_ARG, "hdet_create: cfg and out must not be NULL");
+  WorkPlan work;
+  if (const int rc = plan_work(cfg, tensors, n_tensors, work)) return rc;
+  const std::vector<TensorDesc>& descs = work.descs;
+  const std::vector<Tile>& tiles = work.tiles;
+  const int64_t n_shared_state = work.n_shared_state, partial_numel = work.partial_numel;
+  const int n = cfg->n_replicas;
+  const bool sharded = cfg->n_replicas_global != 0;
+  const int n_global = sharded ? cfg->n_replicas_global : n;
+
   hdet_ctx* h = new (std::nothrow) hdet_ctx();
   if (!h) return fail(nullptr, HDET_ERR_INVALID_ARG, "hdet_create: out of host memory");
   h->cfg = *cfg;
@@ -348,7 +372,29 @@ int hdet_create(const hdet_config* cfg, const hdet_tensor* tensors, int64_t n_te
   return HDET_OK;
 }
 
+int hdet_plan_tiles(const hdet_config* cfg, const hdet_tensor* tensors, int64_t n_tensors, int32_t* tile_tensor,
+                    int32_t* tile_index, int64_t capacity, int64_t* n_tiles, int32_t* tensor_access,
+                    int64_t* partial_offsets) {
+  if (!cfg || !n_tiles) return fail(nullptr, HDET_ERR_INVALID_ARG, "hdet_plan_tiles: cfg and n_tiles must not be NULL");
+  WorkPlan work;
+  if (const int rc = plan_work(cfg, tensors, n_tensors, work)) return rc;
+  *n_tiles = (int64_t)work.tiles.size();
+  if (tile_tensor && tile_index) {
+    if (capacity < *n_tiles) return fail(nullptr, HDET_ERR_INVALID_ARG, "hdet_plan_tiles: capacity is smaller than the tile count");
+    for (size_t i = 0; i < work.tiles.size(); ++i) {
+      tile_tensor[i] = work.tiles[i].tensor;
+      tile_index[i] = work.tiles[i].tile;
+    }
+  }
+  for (int64_t k = 0; k < n_tensors; ++k) {
+    if (tensor_access) tensor_access[k] = work.descs[k].vec;
+    if (partial_offsets) partial_offsets[k] = work.descs[k].partial_off;
+  }
+  return HDET_OK;
+}
+
 int hdet_set_schedule(hdet_handle h, const hdet_schedule* s) {
+  TraceRange trace("hdet_set_schedule");
   if (!h) return HDET_ERR_INVALID_ARG;
   if (!s || !s->max_lr) return fail(h, HDET_ERR_INVALID_ARG, "hdet_set_schedule: sched and max_lr must not be NULL");
   if (h->device_mode)
@@ -462,11 +508,13 @@ static int step_impl(hdet_handle h, const double* step_losses, bool sharded_call
 }
 
 int hdet_step(hdet_handle h, const double* step_losses, void* stream, int32_t* did_converge) {
+  TraceRange trace("hdet_step");
   return step_impl(h, step_losses, false, nullptr, stream, did_converge);
 }
 
 int hdet_step_host_grads(hdet_handle h, const void* const* host_grads, const double* step_losses, void* stream,
                          int32_t* did_converge) {
+  TraceRange trace("hdet_step_host_grads");
   if (!h) return HDET_ERR_INVALID_ARG;
   if (did_converge) *did_converge = 0;
   if (h->n_tensors > 0 && !host_grads) return fail(h, HDET_ERR_INVALID_ARG, "hdet_step_host_grads: host_grads is NULL");
@@ -494,6 +542,7 @@ int hdet_step_host_grads(hdet_handle h, const void* const* host_grads, const dou
 }
 
 int hdet_step_sharded(hdet_handle h, const double* step_losses, void* d_partial, void* stream, int32_t* did_converge) {
+  TraceRange trace("hdet_step_sharded");
   if (!h) return HDET_ERR_INVALID_ARG;
   if (h->n_tiles > 0 && !d_partial) return fail(h, HDET_ERR_INVALID_ARG, "hdet_step_sharded: d_partial is NULL");
   if (d_partial && !aligned(d_partial, 16))
@@ -502,6 +551,7 @@ int hdet_step_sharded(hdet_handle h, const double* step_losses, void* d_partial,
 }
 
 int hdet_apply_mean(hdet_handle h, const void* d_sum, void* stream) {
+  TraceRange trace("hdet_apply_mean");
   if (!h) return HDET_ERR_INVALID_ARG;
   if (h->n_tiles == 0) return HDET_OK;
   if (!d_sum || !aligned(d_sum, 16)) return fail(h, HDET_ERR_INVALID_ARG, "hdet_apply_mean: d_sum is NULL or not 16-byte aligned");
@@ -526,6 +576,7 @@ int hdet_partial_layout(hdet_handle h, int64_t* offsets, int64_t n_offsets, int6
 }
 
 int hdet_step_device(hdet_handle h, const void* d_step_losses, int32_t loss_dtype, void* stream, int32_t* did_converge) {
+  TraceRange trace("hdet_step_device");
   if (!h) return HDET_ERR_INVALID_ARG;
   if (did_converge) *did_converge = 0;
   if (!h->has_schedule) return fail(h, HDET_ERR_STATE, "hdet_step_device: call hdet_set_schedule first");
@@ -583,6 +634,7 @@ int hdet_step_device(hdet_handle h, const void* d_step_losses, int32_t loss_dtyp
 }
 
 int hdet_warm_init(hdet_handle h, double nu, uint64_t seed, void* stream) {
+  TraceRange trace("hdet_warm_init");
   if (!h) return HDET_ERR_INVALID_ARG;
   if (!(nu >= 0.0) || !std::isfinite(nu)) return fail(h, HDET_ERR_INVALID_ARG, "hdet_warm_init: nu must be finite and >= 0");
   if (h->n_tiles == 0) return HDET_OK;
@@ -601,6 +653,7 @@ int hdet_warm_init(hdet_handle h, double nu, uint64_t seed, void* stream) {
 }
 
 int hdet_converge(hdet_handle h, void* stream) {
+  TraceRange trace("hdet_converge");
   if (!h) return HDET_ERR_INVALID_ARG;
   if (h->n_global != h->cfg.n_replicas)
     return fail(h, HDET_ERR_UNSUPPORTED, "hdet_converge: this handle holds a shard of the replica axis; use hdet_step_sharded and hdet_apply_mean");
@@ -615,6 +668,7 @@ int hdet_converge(hdet_handle h, void* stream) {
 }
 
 int hdet_autolr_update(hdet_handle h, const double* round_losses, void* /*stream*/) {
+  TraceRange trace("hdet_autolr_update");
   if (!h) return HDET_ERR_INVALID_ARG;
   if (!h->has_schedule) return fail(h, HDET_ERR_STATE, "hdet_autolr_update: call hdet_set_schedule first");
   if (h->device_mode)
@@ -669,6 +723,7 @@ int hdet_autolr_update(hdet_handle h, const double* round_losses, void* /*stream
 }
 
 int hdet_get_state(hdet_handle h, hdet_state* out) {
+  TraceRange trace("hdet_get_state");
   if (!h) return HDET_ERR_INVALID_ARG;
   if (!out) return fail(h, HDET_ERR_INVALID_ARG, "hdet_get_state: out is NULL");
   if (h->device_mode) {
@@ -695,6 +750,7 @@ int hdet_get_state(hdet_handle h, hdet_state* out) {
 }
 
 int hdet_set_state(hdet_handle h, const hdet_state* in) {
+  TraceRange trace("hdet_set_state");
   if (!h) return HDET_ERR_INVALID_ARG;
   if (!in) return fail(h, HDET_ERR_INVALID_ARG, "hdet_set_state: in is NULL");
   if (in->step < 0 || in->n_acc < 0) return fail(h, HDET_ERR_INVALID_ARG, "hdet_set_state: negative step or n_acc");
@@ -730,6 +786,7 @@ int hdet_set_state(hdet_handle h, const hdet_state* in) {
 }
 
 int hdet_destroy(hdet_handle h) {
+  TraceRange trace("hdet_destroy");
   if (!h) return HDET_OK;
   if (h->d_tensors || h->d_tiles || h->d_status || h->d_state || h->d_warm) {
     DeviceScope scope(h->cfg.device);

@@ -80,6 +80,7 @@ int fail(int code, const char* msg) {
 
 extern "C" HDET_API int hdet_converge_static(const hdet_tensor* tensors, int64_t n_tensors, int32_t n_replicas,
                                              int32_t device, void* stream) {
+  hdet::TraceRange trace("hdet_converge_static");
   if (n_tensors < 0 || (n_tensors > 0 && !tensors))
     return fail(HDET_ERR_INVALID_ARG, "hdet_converge_static: tensors is NULL or n_tensors < 0");
   if (n_replicas < 1 || n_replicas > HDET_MAX_REPLICAS)

@@ -290,3 +290,71 @@ def test_arena_refuses_to_run_without_a_device():
     with pytest.raises(B.HdetError) as e:
         B.hdet_create(cfg, [t])
     assert e.value.status == B.HDET_ERR_CUDA
+
+
+def _fake_descriptors(w, grad_misalign=0):
+    """Descriptors of the workload's tensors laid out like a stacked arena at fake addresses (never dereferenced)."""
+    from hdet_inputs import workloads as W
+    gsz = 2 if w.grad_dtype == W.DTYPE_BF16 else 4
+    offs, p_pad = w.arena_offsets(), w.arena_numel()
+    base = {"param": 0x7000_0000_0000, "grad": 0x7100_0000_0000 + grad_misalign, "m": 0x7200_0000_0000, "v": 0x7300_0000_0000}
+    out = []
+    for t, off in zip(w.tensors, offs):
+        d = B.hdet_tensor(param=base["param"] + 4 * off, grad=base["grad"] + gsz * off, numel=t.numel,
+                          param_stride=p_pad, grad_stride=p_pad, state_stride=p_pad, group=t.group)
+        if w.optimizer == W.OPT_ADAMW:
+            d.exp_avg, d.exp_avg_sq = base["m"] + 4 * off, base["v"] + 4 * off
+        out.append(d)
+    return out
+
+
+@pytest.mark.parametrize("name", ["config1", "config2", "config3", "config4", "config5", "ragged8", "ragged4", "ragged1"])
+def test_work_plan_covers_every_element_of_every_tensor_exactly_once(name):
+    """Walks the tile table hdet_create builds (host arithmetic only): tiles of 2048 elements, tensor by tensor in
+    order, no gap, no overlap, the last tile of a tensor ragged; the access path follows the alignment; the
+    partial-sum offsets do not overlap."""
+    from hdet_inputs import workloads as W
+    from paper_2604_24708_b200 import from_workload
+    w = {"ragged8": lambda: W.ragged_workload(align_elems=8), "ragged4": lambda: W.ragged_workload(align_elems=4),
+         "ragged1": lambda: W.ragged_workload(align_elems=1)}.get(name, W.ALL_CONFIGS.get(name))()
+    descs = _fake_descriptors(w)
+    tt, ti, access, poffs = B.hdet_plan_tiles(from_workload.config_for(w), descs)
+    covered = np.zeros(len(w.tensors), dtype=np.int64)
+    expect_next = {}
+    for k, j in zip(tt, ti):
+        assert j == expect_next.get(k, 0)                       # tiles of a tensor come in order, none skipped or repeated
+        expect_next[k] = j + 1
+        lo, hi = 2048 * j, min(w.tensors[k].numel, 2048 * (j + 1))
+        assert lo < hi
+        covered[k] += hi - lo
+    assert tt == sorted(tt)                                      # tensor by tensor
+    assert covered.tolist() == [t.numel for t in w.tensors]      # every element exactly once
+    assert len(tt) == sum((t.numel + 2047) // 2048 for t in w.tensors)
+    gsz = 2 if w.grad_dtype == W.DTYPE_BF16 else 4
+    adam = w.optimizer == W.OPT_ADAMW
+    for d, a in zip(descs, access):
+        vec = d.param % 16 == 0 and d.grad % (4 * gsz) == 0
+        if adam:
+            vec = vec and d.exp_avg % 16 == 0 and d.exp_avg_sq % 16 == 0
+        bulk = vec and adam and d.grad % 16 == 0 and (d.grad_stride * gsz) % 16 == 0
+        assert a == (3 if bulk else 1 if vec else 0)
+    ends = [o + (t.numel + 3) // 4 * 4 for o, t in zip(poffs, w.tensors)]
+    assert poffs[0] == 0 and all(o % 4 == 0 for o in poffs) and poffs[1:] == ends[:-1]
+
+
+def test_work_plan_rejects_what_create_rejects_and_reports_small_capacity():
+    from hdet_inputs import workloads as W
+    from paper_2604_24708_b200 import from_workload
+    w = W.config2()
+    descs = _fake_descriptors(w)
+    descs[3].numel = 0
+    with pytest.raises(B.HdetError) as e:
+        B.hdet_plan_tiles(from_workload.config_for(w), descs)
+    assert e.value.status == B.HDET_ERR_INVALID_ARG and "tensor 3" in e.value.message
+    descs = _fake_descriptors(w)
+    count = C.c_int64(0)
+    arr = (B.hdet_tensor * len(descs))(*descs)
+    buf = (C.c_int32 * 4)()
+    cfg = from_workload.config_for(w)
+    assert B._lib.hdet_plan_tiles(C.byref(cfg), arr, len(descs), buf, buf, 4, C.byref(count), None, None) == B.HDET_ERR_INVALID_ARG
+    assert count.value == sum((t.numel + 2047) // 2048 for t in w.tensors)
