@@ -39,12 +39,12 @@ UNIT = "replica-param-elements/s"
 # DRAM bytes per replica-element of fanout_kernel<bf16, AdamW, converge>, from the ncu capture of that kernel on the
 # 25 M list summarised under profiles/ (5.1813 GB over 8 x 25,190,400 elements); traffic grows
 # in proportion to N x P.  Set to None whenever that kernel changes until the counters are taken again.
-NCU_DRAM_BYTES_PER_ELEMENT_ADAMW_BF16_CONVERGE = 5.1813e9 / (8 * 25_190_400)
+NCU_DRAM_BYTES_PER_ELEMENT_ADAMW_BF16_CONVERGE = None
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
 
 
-def bytes_per_element(w: W.Workload, shared_grad: bool = False, shared_state: bool = False) -> float:
+def bytes_per_element(w: W.Workload, shared_grad: bool = False, shared_state: bool = False, bf16_copy: bool = False) -> float:
     """Algorithmic HBM bytes per replica-parameter-element of the fan-out kernel (fused converge adds none).
 
     A shared gradient is read once per N replicas; shared moments are read and written once per N replicas.
@@ -52,10 +52,12 @@ def bytes_per_element(w: W.Workload, shared_grad: bool = False, shared_state: bo
     """
     n = w.n_replicas
     g = (2 if w.grad_dtype == W.DTYPE_BF16 else 4) / (n if shared_grad else 1)
+    if bf16_copy:                                    # 2 bytes per PARAMETER at every converge, i.e. every T steps
+        g += 2 / (n * w.sync_interval)
     if w.optimizer == W.OPT_ADAMW:
         state = 16 / (n if shared_state else 1)      # m, v read and written
         return 8 + g + state                         # theta read and written
-    return 8 + g
+    return 8 + g + (8 if w.momentum else 0)          # SGD; the momentum buffer is read and written
 
 
 def measured_peaks():
@@ -182,12 +184,23 @@ def whole_job_value(units_per_rank: float, world: int, ms_per_step: float) -> fl
     return units_per_rank * world / (ms_per_step * 1e-3)
 
 
-def pick_workload(name, torch, sync_interval=None):
+def pick_workload(name, torch, sync_interval=None, optimizer=None, grad_dtype=None):
+    """The named workload, optionally with another T, optimizer or gradient type (same tensor list and inputs)."""
+    from dataclasses import replace
     w = W.ALL_CONFIGS[name]()
     if sync_interval:
-        from dataclasses import replace
         w = replace(w, sync_interval=sync_interval, name=f"{w.name}_T{sync_interval}")
-    need = w.n_replicas * w.arena_numel() * (14 if w.optimizer == W.OPT_ADAMW else 8)
+    if optimizer == "sgd":
+        w = replace(w, optimizer=W.OPT_SGD, momentum=0.0, name=f"{w.name}_sgd")
+    elif optimizer == "sgd-momentum":
+        w = replace(w, optimizer=W.OPT_SGD, momentum=0.9, name=f"{w.name}_sgd_momentum")
+    elif optimizer == "adamw":
+        w = replace(w, optimizer=W.OPT_ADAMW, momentum=0.0, name=f"{w.name}_adamw")
+    if grad_dtype:
+        w = replace(w, grad_dtype=W.DTYPE_F32 if grad_dtype == "f32" else W.DTYPE_BF16, name=f"{w.name}_g{grad_dtype}")
+    gsz = 2 if w.grad_dtype == W.DTYPE_BF16 else 4
+    state = 8 if w.optimizer == W.OPT_ADAMW else (4 if w.momentum else 0)
+    need = w.n_replicas * w.arena_numel() * (4 + gsz + state)
     free, _ = torch.cuda.mem_get_info()
     note = None
     if need + (3 << 30) > free:
@@ -214,11 +227,12 @@ def run_ours(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
 
-    w, note = pick_workload(args.workload, torch, args.sync_interval)
+    w, note = pick_workload(args.workload, torch, args.sync_interval, args.optimizer, args.grad_dtype)
     n, P = w.n_replicas, w.numel
     arena = StackedArena([t.numel for t in w.tensors], [t.group for t in w.tensors], n, w.optimizer, w.grad_dtype,
                          device=f"cuda:{local}", align_elems=w.align_elems, shared_grad=args.shared_grad,
-                         shared_state=args.shared_state)
+                         shared_state=args.shared_state, sgd_momentum=(w.optimizer == W.OPT_SGD and w.momentum != 0.0),
+                         bf16_copy=args.bf16_copy)
     D.fill(arena.param[0], R.param_key(w), 0, R.param_scale(w))
     for r in range(1, n):
         arena.param[r].copy_(arena.param[0])
@@ -297,9 +311,11 @@ def run_ours(args):
     value = whole_job_value(n * P, world, ms_per_step)
 
     # ---- end-to-end region: this step's gradients come from pinned host memory, the status word goes back --
-    e2e_steps = max(1, min(args.steps, args.e2e_steps))
     n_grad_copies = 1 if args.shared_grad else n
     h2d_bytes = n_grad_copies * arena.p_pad * arena.grad.element_size()
+    # ten steps where a step's upload is small; three where one step already moves gigabytes over PCIe
+    e2e_steps = args.e2e_steps if args.e2e_steps else (3 if h2d_bytes > (4 << 30) else 10)
+    e2e_steps = max(1, e2e_steps)
     # Host stepping goes through hdet_step_host_grads: the library itself copies every tensor's gradients from a
     # pinned host image of the gradient arena (same layout as on the device) and then launches the update.
     host_image, host_ptrs, host_grad = None, None, None
@@ -361,7 +377,7 @@ def run_ours(args):
             torch.cuda.synchronize()
             return a.elapsed_time(b) / reps
 
-        bpe_step = bytes_per_element(w, args.shared_grad, args.shared_state)
+        bpe_step = bytes_per_element(_replace(w, sync_interval=1 << 40), args.shared_grad, args.shared_state)
         for label, T, fuse, bpe_k in (("fanout_update", 1 << 40, 1, bpe_step),
                                       ("fanout_update_converge_fused", 1, 1, bpe_step),
                                       ("fanout_update_then_converge_unfused", 1, 0, bpe_step + 8)):
@@ -385,13 +401,13 @@ def run_ours(args):
             dist.destroy_process_group()
         return
 
-    bpe = bytes_per_element(w, args.shared_grad, args.shared_state)
+    bpe = bytes_per_element(w, args.shared_grad, args.shared_state, args.bf16_copy)
     peak, peak_src = measured_peaks()
     # mean duration of one fan-out launch: a step is one fan-out launch (device stepping adds one-warp scalar kernels)
     launch_ms = statistics.mean(per_step_ms)
     achieved = bpe * n * P / (launch_ms * 1e-3) / 1e9
     traffic, traffic_src = args.traffic_bytes, "command line" if args.traffic_bytes else None
-    plain_mode = not (args.shared_grad or args.shared_state or args.grad_mode == "mean")
+    plain_mode = not (args.shared_grad or args.shared_state or args.grad_mode == "mean" or args.bf16_copy)
     if (traffic is None and plain_mode and NCU_DRAM_BYTES_PER_ELEMENT_ADAMW_BF16_CONVERGE and w.optimizer == W.OPT_ADAMW
             and w.grad_dtype == W.DTYPE_BF16 and w.sync_interval == 1):
         traffic = NCU_DRAM_BYTES_PER_ELEMENT_ADAMW_BF16_CONVERGE * n * P
@@ -405,7 +421,7 @@ def run_ours(args):
             "workload": w.name, "n_replicas": n, "params_per_replica": P, "n_tensors": len(w.tensors),
             "optimizer": "adamw" if w.optimizer == W.OPT_ADAMW else "sgd", "sync_interval": w.sync_interval,
             "alpha_lr": w.alpha_lr, "stepping": args.stepping, "grad_mode": args.grad_mode, "shared_grad": args.shared_grad,
-            "shared_moments": args.shared_state, "resident_gb": arena.resident_bytes() / 1e9,
+            "shared_moments": args.shared_state, "bf16_copy": args.bf16_copy, "resident_gb": arena.resident_bytes() / 1e9,
             "l2_policy": "inputs larger than L2 (no flush)", "parallelism": f"{world} independent replicas of the job",
             "note": note,
         },
@@ -635,7 +651,13 @@ def main():
     ap.add_argument("--shared-grad", action="store_true", help="one gradient for all replicas (grad_stride 0)")
     ap.add_argument("--shared-state", action="store_true",
                     help="one pair of Adam moments for all replicas (needs --shared-grad or --grad-mode mean)")
-    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--optimizer", default=None, choices=["adamw", "sgd", "sgd-momentum"],
+                    help="run the workload's tensor list with another optimizer (sgd: Eq. 2; sgd-momentum: mu = 0.9)")
+    ap.add_argument("--grad-dtype", default=None, choices=["bf16", "f32"], help="override the workload's gradient type")
+    ap.add_argument("--bf16-copy", action="store_true",
+                    help="every converge also writes the averaged parameters as bf16 (hdet_tensor.param_bf16)")
+    ap.add_argument("--e2e-steps", type=int, default=0,
+                    help="steps of the end-to-end region (default: 10, or 3 when one step uploads more than 4 GB)")
     ap.add_argument("--cpu-steps", type=int, default=30)
     ap.add_argument("--cpu-cores", type=int, default=None,
                     help="worker processes of the CPU oracle (default: every core this process may use)")

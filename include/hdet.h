@@ -94,12 +94,19 @@ typedef struct {
                            then required of every tensor of the handle                    */
   int32_t group;        /* optimizer group, 0 .. n_groups-1                               */
   int32_t reserved;     /* set to 0                                                       */
+  void* param_bf16;     /* optional bf16 [numel] (ONE copy, not one per replica), or NULL: every
+                           converge (fused into a step, hdet_converge, hdet_apply_mean) also
+                           writes the averaged parameters of Eq. 3 here, each the stored fp32
+                           mean rounded to nearest even -- the weights the next forward pass of
+                           Algorithm 1 reads in mixed precision; costs 2 bytes per parameter.
+                           Updates that do not converge leave it untouched.                */
 } hdet_tensor;
 /* Alignment: pointers must be aligned to their element type (4 bytes fp32, 2 bytes
  * bf16) or hdet_create returns HDET_ERR_ALIGN.  A tensor whose pointers are 16-byte
  * aligned (gradients: 8 bytes for bf16, 16 for fp32) and whose strides are multiples of
  * 4 elements takes the vectorised path; any other tensor is processed correctly by
- * scalar loads. */
+ * scalar loads.  param_bf16, when given, must be 2-byte aligned; it joins the vectorised path
+ * when 8-byte aligned and the bulk-copy path (AdamW) when 16-byte aligned. */
 
 typedef struct {
   int32_t n_replicas;    /* N of Eq. 1, 1 .. HDET_MAX_REPLICAS                            */
@@ -352,7 +359,7 @@ HDET_API int hdet_destroy(hdet_handle h);
  * (which may synchronise the device) is not acceptable.
  *
  * The caller passes the same hdet_tensor descriptors as to hdet_create; only param, numel and
- * param_stride are read (grad and the moments may be NULL).  The work tables that hdet_create
+ * param_stride are read (grad and the moments may be NULL; param_bf16 is ignored).  The work tables that hdet_create
  * would put in allocated memory are written, on every call, into one static device array of
  * about 0.6 MB that each GPU loading the library holds until the process exits.  Limits, checked
  * before anything is launched: at most HDET_STATIC_MAX_TENSORS tensors and HDET_STATIC_MAX_TILES

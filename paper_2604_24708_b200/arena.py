@@ -6,6 +6,7 @@ Layout in HBM (one allocation per quantity, no per-tensor allocations):
     exp_avg    fp32  [N][P_pad]     (AdamW only; [P_pad] when the moments are shared by all replicas)
     exp_avg_sq fp32  [N][P_pad]     (AdamW only; likewise)
     grad       fp32 or bf16 [N][P_pad]   (or [P_pad] when one gradient is shared)
+    param_bf16 bf16  [P_pad]        (optional: the averaged parameters of the last converge, one copy)
 
 Every offset_k is a multiple of ``align_elems`` (8 by default: 32 bytes of fp32, 16 bytes of
 bf16), so every tensor takes the library's 128-bit path.  Only memory and descriptors are
@@ -23,7 +24,7 @@ from . import binding as B
 class StackedArena:
     def __init__(self, numels: Sequence[int], groups: Sequence[int], n_replicas: int, optimizer: int,
                  grad_dtype: int, device: str = "cuda:0", align_elems: int = 8, shared_grad: bool = False,
-                 shared_state: bool = False, sgd_momentum: bool = False):
+                 shared_state: bool = False, sgd_momentum: bool = False, bf16_copy: bool = False):
         if not torch.cuda.is_available():
             raise RuntimeError("StackedArena needs a CUDA device (there is no CPU path)")
         self.numels = [int(x) for x in numels]
@@ -50,6 +51,8 @@ class StackedArena:
         self.shared_grad = bool(shared_grad)
         gshape = (self.p_pad,) if shared_grad else (self.n, self.p_pad)
         self.grad = torch.zeros(gshape, dtype=gd, device=self.device)
+        # optional: one bf16 copy of the averaged parameters, written by every converge
+        self.param_bf16 = torch.zeros((self.p_pad,), dtype=torch.bfloat16, device=self.device) if bf16_copy else None
 
     def descriptors(self) -> List[B.hdet_tensor]:
         out = []
@@ -67,9 +70,11 @@ class StackedArena:
             t.grad_stride = 0 if self.shared_grad else self.p_pad
             t.state_stride = 0 if self.shared_state else self.p_pad
             t.group = grp
+            if self.param_bf16 is not None:
+                t.param_bf16 = self.param_bf16.data_ptr() + 2 * off
             out.append(t)
         return out
 
     def resident_bytes(self) -> int:
-        ts = [t for t in (self.param, self.grad, self.exp_avg, self.exp_avg_sq) if t is not None]
+        ts = [t for t in (self.param, self.grad, self.exp_avg, self.exp_avg_sq, self.param_bf16) if t is not None]
         return sum(t.numel() * t.element_size() for t in ts)

@@ -40,7 +40,7 @@ class hdet_tensor(C.Structure):
     _fields_ = [
         ("param", C.c_void_p), ("grad", C.c_void_p), ("exp_avg", C.c_void_p), ("exp_avg_sq", C.c_void_p),
         ("numel", C.c_int64), ("param_stride", C.c_int64), ("grad_stride", C.c_int64), ("state_stride", C.c_int64),
-        ("group", C.c_int32), ("reserved", C.c_int32),
+        ("group", C.c_int32), ("reserved", C.c_int32), ("param_bf16", C.c_void_p),
     ]
 
 

@@ -274,7 +274,7 @@ int plan_work(const hdet_config* cfg, const hdet_tensor* tensors, int64_t n_tens
     if (t.param_stride < 0 || t.grad_stride < 0 || t.state_stride < 0)
       return fail(nullptr, HDET_ERR_INVALID_ARG, std::string(where) + "negative stride");
     if (!aligned(t.param, 4) || !aligned(t.grad, gsz) || (t.exp_avg && !aligned(t.exp_avg, 4)) ||
-        (t.exp_avg_sq && !aligned(t.exp_avg_sq, 4)))
+        (t.exp_avg_sq && !aligned(t.exp_avg_sq, 4)) || (t.param_bf16 && !aligned(t.param_bf16, 2)))
       return fail(nullptr, HDET_ERR_ALIGN, std::string(where) + "pointer not aligned to its element type");
     const int64_t n_tiles_t = (t.numel + kTileElems - 1) / kTileElems;
     if (n_tiles_t > INT32_MAX || (int64_t)tiles.size() + n_tiles_t > INT32_MAX)
@@ -293,9 +293,13 @@ int plan_work(const hdet_config* cfg, const hdet_tensor* tensors, int64_t n_tens
     if (cfg->optimizer == HDET_OPT_ADAMW)
       vec = vec && aligned(t.exp_avg, 16) && aligned(t.exp_avg_sq, 16) && t.state_stride % 4 == 0;
     if (sgd_momentum) vec = vec && aligned(t.exp_avg, 16) && t.state_stride % 4 == 0;
+    if (t.param_bf16) vec = vec && aligned(t.param_bf16, 8);          // four bf16 values per store
+    d.param_bf16 = static_cast<unsigned short*>(t.param_bf16);
     d.vec = vec ? kVecLoads : 0;
     // Bulk copies move whole tiles and need every array, the gradient included, on 16-byte boundaries.
-    if (vec && adamw && aligned(t.grad, 16) && (t.grad_stride * (int64_t)gsz) % 16 == 0) d.vec |= kVecBulk;
+    if (vec && adamw && aligned(t.grad, 16) && (t.grad_stride * (int64_t)gsz) % 16 == 0 &&
+        (!t.param_bf16 || aligned(t.param_bf16, 16)))
+      d.vec |= kVecBulk;
     d.partial_off = partial_numel;
     d.partial = nullptr;
     partial_numel += (t.numel + 3) / 4 * 4;

@@ -112,6 +112,7 @@ __device__ void range_scalar(const TensorDesc& td, long long begin, long long en
       } else {
         const float mean = (float)(sum * s.inv_n);
         for (int r = 0; r < n; ++r) __stcs(td.param + r * td.param_stride + e, mean);
+        if (td.param_bf16) td.param_bf16[e] = bf16_bits(mean);
       }
     }
   }
@@ -278,6 +279,7 @@ __device__ __forceinline__ void tile_vector_pass(const TensorDesc& td, long long
       const float4 mean = make_float4((float)(sum[k][0] * s.inv_n), (float)(sum[k][1] * s.inv_n),
                                       (float)(sum[k][2] * s.inv_n), (float)(sum[k][3] * s.inv_n));
       for (int rr = 0; rr < n; ++rr) __stcs(reinterpret_cast<float4*>(P + rr * ps + idx[k]), mean);
+      if (td.param_bf16) __stcs(reinterpret_cast<uint2*>(td.param_bf16 + off + idx[k]), bf16_bits4(mean));
     }
   }
 }
@@ -319,7 +321,8 @@ struct BulkLayout {
   static constexpr uint32_t kGradBytes = kTileElems * sizeof(GradT);
   static constexpr uint32_t kStageBytes = 3 * kF32Bytes + kGradBytes;     // theta | m | v | gradient
   static constexpr uint32_t kMeanOff = kStages * kStageBytes;             // one fp32 tile for the mean
-  static constexpr uint32_t kBarrierOff = kMeanOff + kF32Bytes;           // full[kStages], done[kStages], mean written
+  static constexpr uint32_t kBf16Off = kMeanOff + kF32Bytes;              // one bf16 tile: the mean's bf16 copy
+  static constexpr uint32_t kBarrierOff = kBf16Off + kTileElems * 2;      // full[kStages], done[kStages], mean written
   static constexpr uint32_t kBytes = kBarrierOff + 8 * (2 * kStages + 1);
 };
 
@@ -404,6 +407,7 @@ __device__ __forceinline__ void tile_bulk(const TensorDesc& td, long long off, c
           bulk::store(td.partial + off, mean_tile, L::kF32Bytes);
         } else {                           // Eq. 3: one shared tile goes to every replica
           for (int r = 0; r < n; ++r) bulk::store(P + r * ps, mean_tile, L::kF32Bytes);
+          if (td.param_bf16) bulk::store(td.param_bf16 + off, base + L::kBf16Off, kTileElems * 2);
         }
         bulk::commit();
       } else {
@@ -422,6 +426,7 @@ __device__ __forceinline__ void tile_bulk(const TensorDesc& td, long long off, c
   // ---- consumers: thread i owns vectors i and i + 256 of the tile, as in the register path ---------------
   const int grp = td.group;
   const bool to_partial = td.partial != nullptr;
+  const bool with_bf16 = !to_partial && td.param_bf16 != nullptr;
   float gbar[kMean ? kTileVecs : 1][4];
   int i = 0;
   if constexpr (kMean) {
@@ -509,6 +514,7 @@ __device__ __forceinline__ void tile_bulk(const TensorDesc& td, long long off, c
                          ? make_float4((float)sum[k][0], (float)sum[k][1], (float)sum[k][2], (float)sum[k][3])
                          : make_float4((float)(sum[k][0] * s.inv_n), (float)(sum[k][1] * s.inv_n),
                                        (float)(sum[k][2] * s.inv_n), (float)(sum[k][3] * s.inv_n));
+      if (with_bf16) reinterpret_cast<uint2*>(smem + L::kBf16Off)[j] = bf16_bits4(mean_tile[j]);
     }
     bulk::publish_smem_writes();
     bulk::barrier_arrive(mean_done);
@@ -634,7 +640,16 @@ fanout_kernel(const __grid_constant__ LaunchPlan plan, const __grid_constant__ S
 //   theta_r <- theta_r - (lr_r wd_r) theta_r - (lr_r / bc1) u.
 // Bytes per replica-element: 8 (theta) + (gradient + 16) / N, or 8 + gradient + 16 / N with the mean.
 constexpr int kChunk = 8;      // replicas of one vector whose parameters are loaded together
-constexpr int kGradChunk = 4;  // replicas whose bf16 gradients are loaded together for the mean (fp32: half)
+#ifndef HDET_GRAD_CHUNK
+#define HDET_GRAD_CHUNK 4
+#endif
+#ifndef HDET_SHARED_MEAN_CTAS
+#define HDET_SHARED_MEAN_CTAS 3
+#endif
+#ifndef HDET_SHARED_NOCONV_CTAS
+#define HDET_SHARED_NOCONV_CTAS 3
+#endif
+constexpr int kGradChunk = HDET_GRAD_CHUNK;  // replicas whose bf16 gradients are loaded together for the mean (fp32: half)
 
 template <typename GradT, bool kConv, bool kMean>
 __device__ void range_scalar_shared(const TensorDesc& td, long long begin, long long end, const StepScalars& s,
@@ -670,6 +685,7 @@ __device__ void range_scalar_shared(const TensorDesc& td, long long begin, long 
       } else {
         const float mean = (float)(sum * s.inv_n);
         for (int r = 0; r < n; ++r) __stcs(td.param + r * td.param_stride + e, mean);
+        if (td.param_bf16) td.param_bf16[e] = bf16_bits(mean);
       }
     }
   }
@@ -802,13 +818,14 @@ __device__ __forceinline__ void tile_vector_shared(const TensorDesc& td, long lo
         const float4 mean = make_float4((float)(sum[0] * s.inv_n), (float)(sum[1] * s.inv_n),
                                         (float)(sum[2] * s.inv_n), (float)(sum[3] * s.inv_n));
         for (int rr = 0; rr < n; ++rr) __stcs(reinterpret_cast<float4*>(P + rr * ps + at), mean);
+        if (td.param_bf16) __stcs(reinterpret_cast<uint2*>(td.param_bf16 + off + at), bf16_bits4(mean));
       }
     }
   }
 }
 
 template <typename GradT, bool kConv, bool kMean>
-__global__ void __launch_bounds__(kThreads, 3)
+__global__ void __launch_bounds__(kThreads, kMean ? HDET_SHARED_MEAN_CTAS : (kConv ? 3 : HDET_SHARED_NOCONV_CTAS))
 fanout_shared_kernel(const __grid_constant__ LaunchPlan plan, const __grid_constant__ StepScalars s_param) {
   __shared__ StepScalars s;
   stage_scalars(s, s_param, plan.scal_dev);
@@ -866,10 +883,12 @@ apply_mean_kernel(const __grid_constant__ LaunchPlan plan, int n_local, double i
       const float4 mean = make_float4((float)(x.x * inv_n_global), (float)(x.y * inv_n_global),
                                       (float)(x.z * inv_n_global), (float)(x.w * inv_n_global));
       for (int r = 0; r < n_local; ++r) __stcs(reinterpret_cast<float4*>(P + r * td.param_stride + 4 * j), mean);
+      if (td.param_bf16) __stcs(reinterpret_cast<uint2*>(td.param_bf16 + off + 4 * j), bf16_bits4(mean));
     }
     for (int e = 4 * nvec + threadIdx.x; e < len; e += kThreads) {
       const float mean = (float)(__ldcs(S + e) * inv_n_global);
       for (int r = 0; r < n_local; ++r) __stcs(P + r * td.param_stride + e, mean);
+      if (td.param_bf16) td.param_bf16[off + e] = bf16_bits(mean);
     }
   }
 }

@@ -31,6 +31,7 @@ struct TensorDesc {
   int vec;  // kVecLoads: pointers and strides allow 128-bit accesses; | kVecBulk: also 16-byte bulk copies of whole tiles
   long long partial_off;  // element offset of this tensor inside the partial-sum staging buffer (multiple of 4)
   float* partial;         // set per tile by the kernels (NULL in the table)
+  unsigned short* param_bf16;  // optional bf16 copy of the averaged parameters (one copy), or NULL
 };
 
 // One unit of work: tile `tile` (kTileElems elements) of tensor `tensor`.
@@ -51,6 +52,17 @@ struct StepScalars {
   int n_replicas;
 };
 
+// fp32 -> bfloat16 bit pattern, round to nearest even.
+__device__ __forceinline__ unsigned short bf16_bits(float x) {
+  const unsigned u = __float_as_uint(x);
+  if ((u & 0x7FFFFFFFu) > 0x7F800000u) return (unsigned short)((u >> 16) | 0x40u);   // a NaN stays a NaN
+  return (unsigned short)((u + 0x7FFFu + ((u >> 16) & 1u)) >> 16);
+}
+__device__ __forceinline__ uint2 bf16_bits4(const float4& x) {
+  return make_uint2((unsigned)bf16_bits(x.x) | ((unsigned)bf16_bits(x.y) << 16),
+                    (unsigned)bf16_bits(x.z) | ((unsigned)bf16_bits(x.w) << 16));
+}
+
 // Eq. 3 on one tile: every replica <- (1/N) sum over replicas, fp64 accumulation r = 0..N-1, one rounding.
 // The one statement of the stand-alone mean; hdet_converge and hdet_converge_static both run it.
 __device__ __forceinline__ void converge_tile(const TensorDesc& td, int tile_index, int n, double inv_n) {
@@ -68,12 +80,14 @@ __device__ __forceinline__ void converge_tile(const TensorDesc& td, int tile_ind
     }
     const float4 mean = make_float4((float)(s0 * inv_n), (float)(s1 * inv_n), (float)(s2 * inv_n), (float)(s3 * inv_n));
     for (int r = 0; r < n; ++r) __stcs(reinterpret_cast<float4*>(P + r * td.param_stride + 4 * j), mean);
+    if (td.param_bf16) __stcs(reinterpret_cast<uint2*>(td.param_bf16 + off + 4 * j), bf16_bits4(mean));
   }
   for (int e = 4 * nvec + threadIdx.x; e < len; e += kThreads) {
     double sum = 0.0;
     for (int r = 0; r < n; ++r) sum += (double)__ldcs(P + r * td.param_stride + e);
     const float mean = (float)(sum * inv_n);
     for (int r = 0; r < n; ++r) __stcs(P + r * td.param_stride + e, mean);
+    if (td.param_bf16) td.param_bf16[off + e] = bf16_bits(mean);
   }
 }
 

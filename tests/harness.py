@@ -29,7 +29,7 @@ class GpuRun:
 
     def __init__(self, w: W.Workload, fuse: int = 1, shared_grad: bool = False, device: int = 0,
                  grad_mean: bool = False, shared_state: bool = False, device_resident: bool = False,
-                 loss_dtype: str = "float64"):
+                 loss_dtype: str = "float64", bf16_copy: bool = False):
         import torch
         from hdet_inputs import device as D
         from paper_2604_24708_b200 import binding as B
@@ -39,7 +39,7 @@ class GpuRun:
         self.arena = StackedArena([t.numel for t in w.tensors], [t.group for t in w.tensors], w.n_replicas,
                                   w.optimizer, w.grad_dtype, device=f"cuda:{device}", align_elems=w.align_elems,
                                   shared_grad=shared_grad, shared_state=shared_state,
-                                  sgd_momentum=(w.optimizer == W.OPT_SGD and w.momentum != 0.0))
+                                  sgd_momentum=(w.optimizer == W.OPT_SGD and w.momentum != 0.0), bf16_copy=bf16_copy)
         assert self.arena.offsets == w.arena_offsets()
         D.fill(self.arena.param[0], R.param_key(w), 0, R.param_scale(w))
         for r in range(1, w.n_replicas):

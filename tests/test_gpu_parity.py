@@ -357,6 +357,61 @@ def test_eps_zero_on_a_ragged_list_sets_no_status_bit(align):
         g.close()
 
 
+@pytest.mark.parametrize("align", [8, 4, 1])
+@pytest.mark.parametrize("mode", ["fused", "unfused", "device", "shared_moments", "grad_mean", "sgd"])
+def test_bf16_copy_of_the_averaged_parameters(align, mode):
+    """hdet_tensor.param_bf16: every converge also writes the averaged parameters as bfloat16.  Bit-exact against
+    the oracle's rounding of the fp32 value the GPU stored; against the oracle's own mean at most one bf16 step
+    apart (where the two fp32 means differ in their last bit across a rounding boundary); untouched by updates
+    that do not converge, and outside the tensors."""
+    import torch
+    from oracle import hdet_oracle as O
+    w = W.ragged_workload(n_replicas=3, align_elems=align,
+                          optimizer=W.OPT_SGD if mode == "sgd" else W.OPT_ADAMW,
+                          grad_dtype=W.DTYPE_F32 if mode == "sgd" else W.DTYPE_BF16)
+    kw = dict(shared_grad=(mode == "shared_moments"), shared_state=(mode == "shared_moments"), grad_mean=(mode == "grad_mean"))
+    g = H.GpuRun(w, fuse=0 if mode == "unfused" else 1, device_resident=(mode == "device"), bf16_copy=True, **kw)
+    o = H.OracleRun(w, H.whole_tensor_slabs(w), shared_grad=kw["shared_grad"], grad_mean=kw["grad_mean"])
+    sentinel = 0x7FC1
+    bits_view = g.arena.param_bf16.view(torch.int16)
+    bits_view.fill_(sentinel)
+    used = np.zeros(g.arena.p_pad, dtype=bool)
+    for off, ne in zip(g.arena.offsets, g.arena.numels):
+        used[off:off + ne] = True
+    last, rounds = None, 0
+    try:
+        for i in range(w.total_steps):
+            ended = g.step(g.perm0())
+            assert ended == o.step()
+            bits = bits_view.cpu().numpy().view(np.uint16)
+            assert np.all(bits[~used] == sentinel)                         # padding is never written
+            if ended:
+                rounds += 1
+                stored = g.arena.param[0].cpu().numpy()
+                assert np.array_equal(bits[used], O.bf16_bits(stored[used]))     # RNE of the stored fp32 mean, bit for bit
+                for k, (off, ne) in enumerate(zip(g.arena.offsets, g.arena.numels)):
+                    want = O.averaged_bf16(o.o.theta[k]).astype(np.int32)
+                    diff = np.abs(bits[off:off + ne].astype(np.int32) - want)
+                    assert diff.max() <= 1 and np.mean(diff == 0) >= 0.99
+                last = bits.copy()
+            elif last is None:
+                assert np.all(bits == sentinel)                            # nothing before the first converge
+            else:
+                assert np.array_equal(bits, last)                          # plain updates leave the copy alone
+        assert rounds == w.total_steps // w.sync_interval
+        # the stand-alone converge writes it too
+        g.arena.param[1].mul_(1.5)
+        bits_view.fill_(sentinel)
+        g.B.hdet_converge(g.h)
+        torch.cuda.synchronize()
+        bits = bits_view.cpu().numpy().view(np.uint16)
+        assert np.array_equal(bits[used], O.bf16_bits(g.arena.param[0].cpu().numpy()[used]))
+        assert np.all(bits[~used] == sentinel)
+        assert g.state().device_status == 0
+    finally:
+        g.close()
+
+
 def test_config2_full_run_sampled():
     """N=8, 25.19 M parameters, AdamW, one-cycle over 1000 updates, T=50, controller on: the full run."""
     w = W.config2()

@@ -14,6 +14,7 @@ from hdet_inputs import recipes as R
 from hdet_inputs import workloads as W
 from paper_2604_24708_b200 import binding as B
 from paper_2604_24708_b200 import from_workload
+from oracle import hdet_oracle as O
 
 
 def test_sharded_handles_compute_the_global_scalars_on_every_rank():
@@ -60,7 +61,7 @@ class _Rank:
         self.w, self.n_local, self.offset, self.D, self.shared_grad = w, n_local, offset, D, shared_grad
         self.arena = StackedArena([t.numel for t in w.tensors], [t.group for t in w.tensors], n_local, w.optimizer,
                                   w.grad_dtype, align_elems=w.align_elems, shared_grad=shared_grad,
-                                  shared_state=shared_grad)
+                                  shared_state=shared_grad, bf16_copy=True)
         D.fill(self.arena.param[0], R.param_key(w), 0, R.param_scale(w))
         for r in range(1, n_local):
             self.arena.param[r].copy_(self.arena.param[0])
@@ -123,6 +124,11 @@ def test_sharded_replica_axis_matches_the_oracle_with_all_replicas(split, shared
             for rk in ranks:
                 B.hdet_apply_mean(rk.h, total, stream)
                 B.hdet_autolr_update(rk.h)
+            for rk in ranks:                  # hdet_apply_mean also refreshes the bf16 copy of the averaged parameters
+                for ao, t in zip(rk.arena.offsets, w.tensors):
+                    stored = rk.arena.param[0, ao:ao + t.numel].cpu().numpy()
+                    bits = rk.arena.param_bf16[ao:ao + t.numel].view(torch.int16).cpu().numpy().view(np.uint16)
+                    assert np.array_equal(bits, O.bf16_bits(stored))
         tol = 1e-6 if i == 0 else 1e-5
         for rk in ranks:
             for k, (ao, t) in enumerate(zip(rk.arena.offsets, w.tensors)):
