@@ -20,6 +20,7 @@
  *   hdet_warm_init         warm noisy initialisation (Eq. 10)
  *   hdet_converge_static   allocation-free variant of hdet_converge
  *   hdet_plan_tiles        host-only view of the work plan (tests, tools)
+ *   hdet_selftest_bounded_wait   makes a kernel's bounded wait run out, to show the timeout status
  *
  * Conventions
  *   - Every tensor pointer is a DEVICE pointer owned by the caller; it must stay
@@ -346,6 +347,18 @@ HDET_API int hdet_get_state(hdet_handle h, hdet_state* out);
  * Errors: INVALID_ARG (NULL, negative step, an array that is not a permutation).
  */
 HDET_API int hdet_set_state(hdet_handle h, const hdet_state* in);
+
+/*
+ * hdet_selftest_bounded_wait -- (no counterpart in the paper: a diagnostic of the library's failure handling.)
+ * The bulk-copy kernels wait for their own copies with a limit of about a second; a copy that never completes
+ * ends as HDET_ERR_TIMEOUT instead of a hung GPU.  This call exercises that path on purpose and without any
+ * fault: it launches a one-CTA kernel that waits, with the same limit, on a barrier that nothing completes.
+ * About a second later (stream order) bit 1 of the device status word is set; hdet_get_state then returns
+ * HDET_ERR_TIMEOUT, update kernels launched while the bit is set leave their tiles untouched, and
+ * hdet_set_state clears the bit, after which the handle steps normally.  The CUDA context stays usable.
+ * Errors: INVALID_ARG, UNSUPPORTED (handle without tensors), CUDA.
+ */
+HDET_API int hdet_selftest_bounded_wait(hdet_handle h, void* stream);
 
 /* hdet_destroy -- frees the work table and the handle.  NULL is accepted. */
 HDET_API int hdet_destroy(hdet_handle h);

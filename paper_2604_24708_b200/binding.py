@@ -120,6 +120,8 @@ def _load() -> C.CDLL:
                                     C.POINTER(C.c_int32), C.c_int64, C.POINTER(C.c_int64), C.POINTER(C.c_int32),
                                     C.POINTER(C.c_int64)]
     lib.hdet_plan_tiles.restype = C.c_int
+    lib.hdet_selftest_bounded_wait.argtypes = [H, C.c_void_p]
+    lib.hdet_selftest_bounded_wait.restype = C.c_int
     for f in ("hdet_create", "hdet_set_schedule", "hdet_step", "hdet_converge", "hdet_autolr_update",
               "hdet_get_state", "hdet_set_state", "hdet_destroy"):
         getattr(lib, f).restype = C.c_int
@@ -262,6 +264,11 @@ def hdet_plan_tiles(cfg: hdet_config, tensors: Sequence[hdet_tensor]):
     return list(tt)[:n], list(ti)[:n], list(acc)[:len(tensors)], list(offs)[:len(tensors)]
 
 
+def hdet_selftest_bounded_wait(h, stream: int = 0) -> None:
+    """Launches a kernel whose bounded wait runs out (about a second): sets the timeout bit of the status word."""
+    _check(_lib.hdet_selftest_bounded_wait(h, C.c_void_p(stream)), h)
+
+
 def hdet_warm_init(h, nu: float = 0.01, seed: int = 0, stream: int = 0) -> None:
     """Eq. 10: every replica <- replica 0 (the checkpoint) + Gaussian noise of relative scale nu."""
     _check(_lib.hdet_warm_init(h, nu, seed, C.c_void_p(stream)), h)
@@ -293,7 +300,7 @@ def hdet_autolr_update(h, round_losses: Optional[Sequence[float]] = None, stream
 def hdet_get_state(h, raise_on_nonfinite: bool = True) -> hdet_state:
     st = hdet_state()
     status = _lib.hdet_get_state(h, C.byref(st))
-    if status == HDET_ERR_NONFINITE and not raise_on_nonfinite:
+    if status in (HDET_ERR_NONFINITE, HDET_ERR_TIMEOUT) and not raise_on_nonfinite:   # sticky device flags: *out is filled
         return st
     _check(status, h)
     return st

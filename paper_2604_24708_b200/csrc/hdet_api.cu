@@ -789,6 +789,18 @@ int hdet_set_state(hdet_handle h, const hdet_state* in) {
   return HDET_OK;
 }
 
+int hdet_selftest_bounded_wait(hdet_handle h, void* stream) {
+  if (!h) return HDET_ERR_INVALID_ARG;
+  TraceRange trace("hdet_selftest_bounded_wait");
+  if (!h->d_status) return fail(h, HDET_ERR_UNSUPPORTED, "hdet_selftest_bounded_wait: the handle has no tensors, hence no device");
+  DeviceScope scope(h->cfg.device);
+  if (scope.err != cudaSuccess) return fail_cuda(h, "hdet_selftest_bounded_wait", scope.err);
+  const cudaError_t e = launch_bounded_wait_probe(h->d_status, static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return fail_cuda(h, "hdet_selftest_bounded_wait: launch", e);
+  ++h->launches;
+  return HDET_OK;
+}
+
 int hdet_destroy(hdet_handle h) {
   TraceRange trace("hdet_destroy");
   if (!h) return HDET_OK;

@@ -46,14 +46,17 @@ __device__ __forceinline__ bool barrier_try_wait(uint32_t bar, uint32_t parity) 
   return done != 0;
 }
 
-// Waits for the phase with the given parity.  Returns false after about a second (2e9 SM cycles).
-__device__ __forceinline__ bool barrier_wait(uint32_t bar, uint32_t parity) {
+// Longest time any wait spins: 2e9 SM cycles, about a second.
+constexpr long long kWaitLimitCycles = 2000000000ll;
+
+// Waits for the phase with the given parity.  Returns false once the limit has passed.
+__device__ __forceinline__ bool barrier_wait(uint32_t bar, uint32_t parity, long long limit_cycles = kWaitLimitCycles) {
   if (barrier_try_wait(bar, parity)) return true;
   const long long start = clock64();
   for (;;) {
     for (int i = 0; i < 32; ++i)
       if (barrier_try_wait(bar, parity)) return true;
-    if (clock64() - start > 2000000000ll) return false;
+    if (clock64() - start > limit_cycles) return false;
   }
 }
 

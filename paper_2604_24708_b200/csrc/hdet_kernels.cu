@@ -640,16 +640,7 @@ fanout_kernel(const __grid_constant__ LaunchPlan plan, const __grid_constant__ S
 //   theta_r <- theta_r - (lr_r wd_r) theta_r - (lr_r / bc1) u.
 // Bytes per replica-element: 8 (theta) + (gradient + 16) / N, or 8 + gradient + 16 / N with the mean.
 constexpr int kChunk = 8;      // replicas of one vector whose parameters are loaded together
-#ifndef HDET_GRAD_CHUNK
-#define HDET_GRAD_CHUNK 4
-#endif
-#ifndef HDET_SHARED_MEAN_CTAS
-#define HDET_SHARED_MEAN_CTAS 3
-#endif
-#ifndef HDET_SHARED_NOCONV_CTAS
-#define HDET_SHARED_NOCONV_CTAS 3
-#endif
-constexpr int kGradChunk = HDET_GRAD_CHUNK;  // replicas whose bf16 gradients are loaded together for the mean (fp32: half)
+constexpr int kGradChunk = 4;  // replicas whose bf16 gradients are loaded together for the mean (fp32: half)
 
 template <typename GradT, bool kConv, bool kMean>
 __device__ void range_scalar_shared(const TensorDesc& td, long long begin, long long end, const StepScalars& s,
@@ -824,8 +815,12 @@ __device__ __forceinline__ void tile_vector_shared(const TensorDesc& td, long lo
   }
 }
 
+// Three CTAs per SM (80 registers).  Six of the eight instantiations then spill 8 - 96 bytes per thread; giving
+// those two CTAs and 128 registers instead removes the spills and measured 2 - 10 % SLOWER on the 1.3 B list
+// (6.26 against 6.63 TB/s for the gradient mean with converge): the third CTA's loads in flight are worth more
+// than the few spilled values, which stay in L1.
 template <typename GradT, bool kConv, bool kMean>
-__global__ void __launch_bounds__(kThreads, kMean ? HDET_SHARED_MEAN_CTAS : (kConv ? 3 : HDET_SHARED_NOCONV_CTAS))
+__global__ void __launch_bounds__(kThreads, 3)
 fanout_shared_kernel(const __grid_constant__ LaunchPlan plan, const __grid_constant__ StepScalars s_param) {
   __shared__ StepScalars s;
   stage_scalars(s, s_param, plan.scal_dev);
@@ -947,6 +942,24 @@ cudaError_t launch_fanout(int optimizer, bool sgd_momentum, int grad_dtype, bool
   if (grad_dtype == HDET_DTYPE_BF16)
     return pick_flags<__nv_bfloat16>(opt, converge, grad_mean, shared_state, plan, s, stream);
   return pick_flags<float>(opt, converge, grad_mean, shared_state, plan, s, stream);
+}
+
+// One CTA waits, with the limit every bulk-copy wait has, on a barrier that nothing will complete, and records
+// the outcome the way tile_bulk does.
+__global__ void bounded_wait_probe_kernel(unsigned* status) {
+  __shared__ __align__(8) unsigned long long barrier;
+  const uint32_t bar = bulk::smem_addr(&barrier);
+  if (threadIdx.x == 0) {
+    bulk::barrier_init(bar, 1);
+    bulk::barrier_init_fence();
+  }
+  __syncthreads();
+  if (!bulk::barrier_wait(bar, 0) && threadIdx.x == 0) atomicOr(status, 2u);
+}
+
+cudaError_t launch_bounded_wait_probe(unsigned* status, cudaStream_t stream) {
+  bounded_wait_probe_kernel<<<1, 32, 0, stream>>>(status);
+  return cudaGetLastError();
 }
 
 cudaError_t launch_apply_mean(const LaunchPlan& plan, int n_local, double inv_n_global, cudaStream_t stream) {

@@ -117,6 +117,9 @@ cudaError_t launch_warm_init(const LaunchPlan& plan, int n_replicas, int replica
 // Every local replica <- plan.partial * inv_n_global (the all-reduced sums of a sharded converge).
 cudaError_t launch_apply_mean(const LaunchPlan& plan, int n_local, double inv_n_global, cudaStream_t stream);
 
+// Diagnostic: a one-CTA kernel whose bounded barrier wait runs out (about a second) and sets bit 1 of *status.
+cudaError_t launch_bounded_wait_probe(unsigned* status, cudaStream_t stream);
+
 // Stand-alone Eq. 3.
 cudaError_t launch_converge(const LaunchPlan& plan, int n_replicas, cudaStream_t stream);
 

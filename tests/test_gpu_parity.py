@@ -412,6 +412,45 @@ def test_bf16_copy_of_the_averaged_parameters(align, mode):
         g.close()
 
 
+def test_a_wait_that_runs_out_becomes_a_status_and_the_context_stays_usable():
+    """Failure handling without a fault: hdet_selftest_bounded_wait makes a kernel wait, with the limit every
+    bulk-copy wait has, on a barrier that nothing completes.  The wait ends by itself after about a second, the
+    status word carries the timeout bit, update kernels launched meanwhile leave the data alone, hdet_set_state
+    clears the bit, and the run then continues in step with the oracle."""
+    import time
+    import torch
+    w = W.ragged_workload(n_replicas=3)
+    g = H.GpuRun(w)
+    o = H.OracleRun(w, H.whole_tensor_slabs(w))
+    try:
+        assert g.step(g.perm0()) == o.step()
+        clean = g.state()
+        before = [g.arena.param.clone(), g.arena.exp_avg.clone(), g.arena.exp_avg_sq.clone()]
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        g.B.hdet_selftest_bounded_wait(g.h, torch.cuda.current_stream().cuda_stream)
+        torch.cuda.synchronize()
+        waited = time.perf_counter() - t0
+        assert 0.3 < waited < 20.0                      # bounded: about 2e9 SM cycles, not forever
+        with pytest.raises(g.B.HdetError) as e:
+            g.B.hdet_get_state(g.h)
+        assert e.value.status == g.B.HDET_ERR_TIMEOUT
+        assert g.B.hdet_get_state(g.h, raise_on_nonfinite=False).device_status & 2
+        g.fill_grads(1)
+        g.B.hdet_step(g.h, None)                        # launched while the bit is set: every CTA leaves at once
+        torch.cuda.synchronize()
+        for a, b in zip(before, [g.arena.param, g.arena.exp_avg, g.arena.exp_avg_sq]):
+            assert torch.equal(a, b)
+        g.B.hdet_set_state(g.h, clean)                  # back to the state after update 1; clears the status word
+        assert g.state().device_status == 0
+        for i in range(1, w.total_steps):
+            assert g.step(g.perm0()) == o.step()
+        H.compare_slabs(g, o, TOL_FULL_RUN)
+        H.compare_scalars(g.state(), o.o, w.n_replicas, w.n_groups)
+    finally:
+        g.close()
+
+
 def test_config2_full_run_sampled():
     """N=8, 25.19 M parameters, AdamW, one-cycle over 1000 updates, T=50, controller on: the full run."""
     w = W.config2()
