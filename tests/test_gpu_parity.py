@@ -358,7 +358,7 @@ def test_eps_zero_on_a_ragged_list_sets_no_status_bit(align):
 
 
 @pytest.mark.parametrize("align", [8, 4, 1])
-@pytest.mark.parametrize("mode", ["fused", "unfused", "device", "shared_moments", "grad_mean", "sgd"])
+@pytest.mark.parametrize("mode", ["fused", "fused_f32_grads", "unfused", "device", "shared_moments", "grad_mean", "sgd"])
 def test_bf16_copy_of_the_averaged_parameters(align, mode):
     """hdet_tensor.param_bf16: every converge also writes the averaged parameters as bfloat16.  Bit-exact against
     the oracle's rounding of the fp32 value the GPU stored; against the oracle's own mean at most one bf16 step
@@ -368,7 +368,7 @@ def test_bf16_copy_of_the_averaged_parameters(align, mode):
     from oracle import hdet_oracle as O
     w = W.ragged_workload(n_replicas=3, align_elems=align,
                           optimizer=W.OPT_SGD if mode == "sgd" else W.OPT_ADAMW,
-                          grad_dtype=W.DTYPE_F32 if mode == "sgd" else W.DTYPE_BF16)
+                          grad_dtype=W.DTYPE_F32 if mode in ("sgd", "fused_f32_grads") else W.DTYPE_BF16)
     kw = dict(shared_grad=(mode == "shared_moments"), shared_state=(mode == "shared_moments"), grad_mean=(mode == "grad_mean"))
     g = H.GpuRun(w, fuse=0 if mode == "unfused" else 1, device_resident=(mode == "device"), bf16_copy=True, **kw)
     o = H.OracleRun(w, H.whole_tensor_slabs(w), shared_grad=kw["shared_grad"], grad_mean=kw["grad_mean"])
