@@ -36,10 +36,10 @@ from hdet_inputs import workloads as W  # noqa: E402
 
 METRIC = "fan-out step+converge throughput (replica-parameter-elements updated per second)"
 UNIT = "replica-param-elements/s"
-# DRAM bytes per replica-element of fanout_kernel<bf16, AdamW, converge>, from the ncu capture of that kernel on the
-# 25 M list summarised under profiles/ (5.1813 GB over 8 x 25,190,400 elements); traffic grows
+# DRAM bytes per replica-element of fanout_kernel<bf16, AdamW, converge> (the bulk-copy kernel), from the ncu capture
+# of that kernel on the 25 M list summarised under profiles/ (5.1818 GB over 8 x 25,190,400 elements); traffic grows
 # in proportion to N x P.  Set to None whenever that kernel changes until the counters are taken again.
-NCU_DRAM_BYTES_PER_ELEMENT_ADAMW_BF16_CONVERGE = None
+NCU_DRAM_BYTES_PER_ELEMENT_ADAMW_BF16_CONVERGE = 5.1818e9 / (8 * 25_190_400)
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
 
