@@ -361,6 +361,8 @@ int hdet_create(const hdet_config* cfg, const hdet_tensor* tensors, int64_t n_te
     if (e == cudaSuccess) e = cudaMemcpy(h->d_tensors, descs.data(), descs.size() * sizeof(TensorDesc), cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemcpy(h->d_tiles, tiles.data(), tiles.size() * sizeof(Tile), cudaMemcpyHostToDevice);
     if (e == cudaSuccess) e = cudaMemset(h->d_status, 0, sizeof(unsigned));
+    if (e == cudaSuccess)
+      e = prepare_fanout(cfg->optimizer, cfg->grad_dtype, cfg->grad_mode == HDET_GRAD_REPLICA_MEAN, h->shared_state);
     if (e != cudaSuccess) {
       free_device(h);
       delete h;

@@ -888,22 +888,37 @@ apply_mean_kernel(const __grid_constant__ LaunchPlan plan, int n_local, double i
   }
 }
 
+// The stage ring needs more dynamic shared memory than the default limit: opt in once per device and kernel.
+template <typename Kernel>
+cudaError_t opt_in_shared_memory(Kernel kernel, int bytes, bool (&opted_in)[kMaxDevices]) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  if (!opted_in[dev]) {
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e != cudaSuccess) return e;
+    opted_in[dev] = true;
+  }
+  return cudaSuccess;
+}
+
+template <typename GradT, int kOpt, bool kConv, bool kMean>
+cudaError_t opt_in_one() {
+  if constexpr (kHasBulkPath<kOpt>) {
+    static bool opted_in[kMaxDevices] = {};
+    return opt_in_shared_memory(fanout_kernel<GradT, kOpt, kConv, kMean>, (int)BulkLayout<GradT>::kBytes, opted_in);
+  }
+  return cudaSuccess;
+}
+
 template <typename GradT, int kOpt, bool kConv, bool kMean>
 cudaError_t launch_one(const LaunchPlan& plan, const StepScalars& s, cudaStream_t stream) {
   if constexpr (kHasBulkPath<kOpt>) {
-    // The stage ring needs more dynamic shared memory than the default limit: opt in once per device.
-    constexpr int kSmem = (int)BulkLayout<GradT>::kBytes;
-    static bool opted_in[kMaxDevices] = {};
-    int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
+    const cudaError_t e = opt_in_one<GradT, kOpt, kConv, kMean>();   // a flag check after the first time
     if (e != cudaSuccess) return e;
-    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
-    if (!opted_in[dev]) {
-      e = cudaFuncSetAttribute(fanout_kernel<GradT, kOpt, kConv, kMean>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
-      if (e != cudaSuccess) return e;
-      opted_in[dev] = true;
-    }
-    fanout_kernel<GradT, kOpt, kConv, kMean><<<plan.n_tiles, kThreads + kProducerThreads, kSmem, stream>>>(plan, s);
+    fanout_kernel<GradT, kOpt, kConv, kMean>
+        <<<plan.n_tiles, kThreads + kProducerThreads, BulkLayout<GradT>::kBytes, stream>>>(plan, s);
   } else {
     fanout_kernel<GradT, kOpt, kConv, kMean><<<plan.grid, kThreads, 0, stream>>>(plan, s);
   }
@@ -934,6 +949,21 @@ cudaError_t pick_flags(int opt, bool converge, bool mean, bool shared_state, con
 }
 
 }  // namespace
+
+cudaError_t prepare_fanout(int optimizer, int grad_dtype, bool grad_mean, bool shared_state) {
+  if (optimizer != HDET_OPT_ADAMW || shared_state) return cudaSuccess;     // only the bulk-copy kernels need it
+  cudaError_t e;
+  if (grad_dtype == HDET_DTYPE_BF16) {
+    e = grad_mean ? opt_in_one<__nv_bfloat16, kOptAdamW, true, true>() : opt_in_one<__nv_bfloat16, kOptAdamW, true, false>();
+    if (e == cudaSuccess)
+      e = grad_mean ? opt_in_one<__nv_bfloat16, kOptAdamW, false, true>() : opt_in_one<__nv_bfloat16, kOptAdamW, false, false>();
+  } else {
+    e = grad_mean ? opt_in_one<float, kOptAdamW, true, true>() : opt_in_one<float, kOptAdamW, true, false>();
+    if (e == cudaSuccess)
+      e = grad_mean ? opt_in_one<float, kOptAdamW, false, true>() : opt_in_one<float, kOptAdamW, false, false>();
+  }
+  return e;
+}
 
 cudaError_t launch_fanout(int optimizer, bool sgd_momentum, int grad_dtype, bool converge, bool grad_mean,
                           bool shared_state, const LaunchPlan& plan, const StepScalars& s, cudaStream_t stream) {

@@ -109,6 +109,10 @@ struct LaunchPlan {
 cudaError_t launch_fanout(int optimizer, bool sgd_momentum, int grad_dtype, bool converge, bool grad_mean,
                           bool shared_state, const LaunchPlan& plan, const StepScalars& s, cudaStream_t stream);
 
+// Per device, before the first launch: lets the bulk-copy kernels this handle will use take their shared-memory
+// ring (an attribute of the kernel).  Called by hdet_create so that no attribute call falls into a stream capture.
+cudaError_t prepare_fanout(int optimizer, int grad_dtype, bool grad_mean, bool shared_state);
+
 // Eq. 10: every replica <- replica 0 + N(0, nu^2 ||replica 0||^2 / total_numel) noise.  `scratch` holds
 // n_tiles + 1 doubles.  Three launches.
 cudaError_t launch_warm_init(const LaunchPlan& plan, int n_replicas, int replica_offset, double nu, double total_numel,

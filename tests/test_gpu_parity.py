@@ -412,6 +412,32 @@ def test_bf16_copy_of_the_averaged_parameters(align, mode):
         g.close()
 
 
+def test_the_first_step_of_a_fresh_handle_can_be_recorded_into_a_cuda_graph():
+    """hdet_create prepares the bulk-copy kernels (their shared-memory attribute), so even the very first
+    hdet_step of a handle makes no attribute call and can be captured; a replay equals a direct step bit for bit."""
+    import torch
+    w = replace(W.ragged_workload(n_replicas=4, numels=(4097, 2048, 33, 12289)), sync_interval=1)
+    direct = H.GpuRun(w)
+    direct.fill_grads(0)
+    direct.B.hdet_step(direct.h, None)
+    torch.cuda.synchronize()
+    g = H.GpuRun(w)
+    g.fill_grads(0)
+    torch.cuda.synchronize()
+    graph, side = torch.cuda.CUDAGraph(), torch.cuda.Stream()
+    with torch.cuda.graph(graph, stream=side):
+        g.B.hdet_step(g.h, None, torch.cuda.current_stream().cuda_stream)      # recorded, not run
+    assert torch.equal(g.arena.exp_avg, torch.zeros_like(g.arena.exp_avg))
+    graph.replay()
+    torch.cuda.synchronize()
+    for a, b in ((g.arena.param, direct.arena.param), (g.arena.exp_avg, direct.arena.exp_avg),
+                 (g.arena.exp_avg_sq, direct.arena.exp_avg_sq)):
+        assert torch.equal(a, b)
+    assert g.state().device_status == 0
+    g.close()
+    direct.close()
+
+
 def test_a_wait_that_runs_out_becomes_a_status_and_the_context_stays_usable():
     """Failure handling without a fault: hdet_selftest_bounded_wait makes a kernel wait, with the limit every
     bulk-copy wait has, on a barrier that nothing completes.  The wait ends by itself after about a second, the
