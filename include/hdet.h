@@ -16,7 +16,7 @@
  * and, around that core:
  *   hdet_step_device       the same step with the scalar state and the controller on the device
  *   hdet_step_host_grads   the same step with the gradients uploaded from host memory first
- *   hdet_step_sharded / hdet_apply_mean / hdet_partial_layout   replica axis split over GPUs
+ *   hdet_step_sharded / hdet_apply_mean / hdet_apply_mean_peers / hdet_partial_layout   replica axis split over GPUs
  *   hdet_warm_init         warm noisy initialisation (Eq. 10)
  *   hdet_converge_static   allocation-free variant of hdet_converge
  *   hdet_plan_tiles        host-only view of the work plan (tests, tools)
@@ -268,6 +268,23 @@ HDET_API int hdet_step_sharded(hdet_handle h, const double* step_losses, void* d
                                int32_t* did_converge);
 HDET_API int hdet_apply_mean(hdet_handle h, const void* d_sum, void* stream);
 HDET_API int hdet_partial_layout(hdet_handle h, int64_t* offsets, int64_t n_offsets, int64_t* total_numel);
+
+/*
+ * hdet_apply_mean_peers -- Eq. 3 across GPUs with the exchange inside the kernel instead of a collective call:
+ * the second half of a sharded converge reads EVERY rank's staging buffer itself.  d_partials is a HOST array of
+ * n_buffers DEVICE pointers, one per rank and in rank order (the same order on every rank, so that every rank
+ * adds the same numbers in the same order and obtains the same bits): this GPU's own d_partial and its peers',
+ * mapped into this process (peer access enabled, CUDA IPC, or symmetric memory) and read with ordinary loads
+ * over NVLink.  Every local replica <- (sum over the buffers, fp64) / N; param_bf16 is refreshed.
+ * The kernel waits for nobody.  The CALLER orders it: (1) every rank's hdet_step_sharded of the round; (2) a
+ * barrier across the ranks that follows those kernels in stream order; (3) this call on every rank; (4) a second
+ * barrier (or a second set of staging buffers used in alternation) before any rank's next round overwrites its
+ * buffer.  Each rank reads (n_buffers - 1) x P floats from its peers, where a ring or in-switch all-reduce moves
+ * 2 (W - 1) / W x P: the same at two ranks, four times as much at eight, so this form suits few ranks or small
+ * models; hdet_apply_mean after an all-reduce is the general one.
+ * Errors: INVALID_ARG (NULL or misaligned buffer, n_buffers outside 1 .. 32), CUDA.
+ */
+HDET_API int hdet_apply_mean_peers(hdet_handle h, const void* const* d_partials, int32_t n_buffers, void* stream);
 
 /*
  * hdet_step_device -- hdet_step and, at the end of a round, hdet_autolr_update, with Algorithm 1's

@@ -101,6 +101,8 @@ def _load() -> C.CDLL:
     lib.hdet_step_sharded.restype = C.c_int
     lib.hdet_apply_mean.argtypes = [H, C.c_void_p, C.c_void_p]
     lib.hdet_apply_mean.restype = C.c_int
+    lib.hdet_apply_mean_peers.argtypes = [H, C.POINTER(C.c_void_p), C.c_int32, C.c_void_p]
+    lib.hdet_apply_mean_peers.restype = C.c_int
     lib.hdet_partial_layout.argtypes = [H, C.POINTER(C.c_int64), C.c_int64, C.POINTER(C.c_int64)]
     lib.hdet_partial_layout.restype = C.c_int
     lib.hdet_warm_init.argtypes = [H, C.c_double, C.c_uint64, C.c_void_p]
@@ -241,6 +243,13 @@ def hdet_step_sharded(h, step_losses, d_partial, stream: int = 0) -> bool:
 
 def hdet_apply_mean(h, d_sum, stream: int = 0) -> None:
     _check(_lib.hdet_apply_mean(h, C.c_void_p(d_sum.data_ptr()), C.c_void_p(stream)), h)
+
+
+def hdet_apply_mean_peers(h, d_partials, stream: int = 0) -> None:
+    """Every local replica <- (sum over the ranks' staging buffers, in the given rank order) / N, read by the kernel itself."""
+    ptrs = [p.data_ptr() if hasattr(p, "data_ptr") else int(p) for p in d_partials]
+    arr = (C.c_void_p * len(ptrs))(*ptrs)
+    _check(_lib.hdet_apply_mean_peers(h, arr, len(ptrs), C.c_void_p(stream)), h)
 
 
 def hdet_partial_layout(h, n_tensors: int):

@@ -571,6 +571,28 @@ int hdet_apply_mean(hdet_handle h, const void* d_sum, void* stream) {
   return HDET_OK;
 }
 
+int hdet_apply_mean_peers(hdet_handle h, const void* const* d_partials, int32_t n_buffers, void* stream) {
+  if (!h) return HDET_ERR_INVALID_ARG;
+  TraceRange trace("hdet_apply_mean_peers");
+  if (h->n_tiles == 0) return HDET_OK;
+  if (!d_partials || n_buffers < 1 || n_buffers > HDET_MAX_REPLICAS)
+    return fail(h, HDET_ERR_INVALID_ARG, "hdet_apply_mean_peers: need 1 .. 32 staging buffers");
+  const float* bufs[HDET_MAX_REPLICAS];
+  for (int b = 0; b < n_buffers; ++b) {
+    if (!d_partials[b] || !aligned(d_partials[b], 16))
+      return fail(h, HDET_ERR_INVALID_ARG, "hdet_apply_mean_peers: a staging buffer is NULL or not 16-byte aligned");
+    bufs[b] = static_cast<const float*>(d_partials[b]);
+  }
+  DeviceScope scope(h->cfg.device);
+  if (scope.err != cudaSuccess) return fail_cuda(h, "hdet_apply_mean_peers", scope.err);
+  LaunchPlan plan{h->d_tensors, h->d_tiles, h->n_tiles, h->grid_converge, h->d_status, nullptr, nullptr};
+  cudaError_t e = launch_apply_mean_peers(plan, bufs, n_buffers, h->cfg.n_replicas, 1.0 / (double)h->n_global,
+                                          static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return fail_cuda(h, "hdet_apply_mean_peers: launch", e);
+  ++h->launches;
+  return HDET_OK;
+}
+
 int hdet_partial_layout(hdet_handle h, int64_t* offsets, int64_t n_offsets, int64_t* total_numel) {
   if (!h) return HDET_ERR_INVALID_ARG;
   if (offsets && n_offsets != h->n_tensors)

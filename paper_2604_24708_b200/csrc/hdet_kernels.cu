@@ -888,6 +888,51 @@ apply_mean_kernel(const __grid_constant__ LaunchPlan plan, int n_local, double i
   }
 }
 
+// ---- the same with the exchange inside the kernel: plain loads from every rank's staging buffer ---------
+// bufs.p[b] is rank b's staging buffer (this GPU's own, or a peer's mapped into this process and read over
+// NVLink with ordinary loads).  The sums are added in rank order b = 0..B-1 in fp64, so every rank computes the
+// same bits; the mean goes to the local replicas.  The kernel waits for nobody: the caller orders it after every
+// rank's hdet_step_sharded (a barrier between the two launches) and keeps the buffers untouched until every
+// rank's launch of this kernel has finished.
+struct PeerBuffers {
+  const float* p[HDET_MAX_REPLICAS];
+  int count;
+};
+
+__global__ void __launch_bounds__(kThreads, 4)
+apply_mean_peers_kernel(const __grid_constant__ LaunchPlan plan, const __grid_constant__ PeerBuffers bufs, int n_local,
+                        double inv_n_global) {
+  for (int t = blockIdx.x; t < plan.n_tiles; t += gridDim.x) {
+    const Tile tile = plan.tiles[t];
+    const TensorDesc td = plan.tensors[tile.tensor];
+    const long long off = (long long)tile.tile * kTileElems;
+    const long long rest = td.numel - off;
+    const int len = rest < kTileElems ? (int)rest : kTileElems;
+    const int nvec = td.vec ? (len >> 2) : 0;
+    float* const P = td.param + off;
+    const long long at = td.partial_off + off;
+    for (int j = threadIdx.x; j < nvec; j += kThreads) {
+      double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
+#pragma unroll 4
+      for (int b = 0; b < bufs.count; ++b) {
+        const float4 x = __ldcs(reinterpret_cast<const float4*>(bufs.p[b] + at + 4 * j));
+        s0 += (double)x.x; s1 += (double)x.y; s2 += (double)x.z; s3 += (double)x.w;
+      }
+      const float4 mean = make_float4((float)(s0 * inv_n_global), (float)(s1 * inv_n_global),
+                                      (float)(s2 * inv_n_global), (float)(s3 * inv_n_global));
+      for (int r = 0; r < n_local; ++r) __stcs(reinterpret_cast<float4*>(P + r * td.param_stride + 4 * j), mean);
+      if (td.param_bf16) __stcs(reinterpret_cast<uint2*>(td.param_bf16 + off + 4 * j), bf16_bits4(mean));
+    }
+    for (int e = 4 * nvec + threadIdx.x; e < len; e += kThreads) {
+      double sum = 0.0;
+      for (int b = 0; b < bufs.count; ++b) sum += (double)__ldcs(bufs.p[b] + at + e);
+      const float mean = (float)(sum * inv_n_global);
+      for (int r = 0; r < n_local; ++r) __stcs(P + r * td.param_stride + e, mean);
+      if (td.param_bf16) td.param_bf16[off + e] = bf16_bits(mean);
+    }
+  }
+}
+
 // The stage ring needs more dynamic shared memory than the default limit: opt in once per device and kernel.
 template <typename Kernel>
 cudaError_t opt_in_shared_memory(Kernel kernel, int bytes, bool (&opted_in)[kMaxDevices]) {
@@ -995,6 +1040,16 @@ cudaError_t launch_bounded_wait_probe(unsigned* status, cudaStream_t stream) {
 cudaError_t launch_apply_mean(const LaunchPlan& plan, int n_local, double inv_n_global, cudaStream_t stream) {
   if (plan.n_tiles == 0) return cudaSuccess;
   apply_mean_kernel<<<plan.grid, kThreads, 0, stream>>>(plan, n_local, inv_n_global);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_apply_mean_peers(const LaunchPlan& plan, const float* const* buffers, int n_buffers, int n_local,
+                                    double inv_n_global, cudaStream_t stream) {
+  if (plan.n_tiles == 0) return cudaSuccess;
+  PeerBuffers bufs{};
+  for (int b = 0; b < n_buffers; ++b) bufs.p[b] = buffers[b];
+  bufs.count = n_buffers;
+  apply_mean_peers_kernel<<<plan.grid, kThreads, 0, stream>>>(plan, bufs, n_local, inv_n_global);
   return cudaGetLastError();
 }
 

@@ -121,6 +121,11 @@ cudaError_t launch_warm_init(const LaunchPlan& plan, int n_replicas, int replica
 // Every local replica <- plan.partial * inv_n_global (the all-reduced sums of a sharded converge).
 cudaError_t launch_apply_mean(const LaunchPlan& plan, int n_local, double inv_n_global, cudaStream_t stream);
 
+// The same with the exchange done by the kernel: every local replica <- (sum over the n_buffers staging buffers,
+// in the given order) * inv_n_global.  The buffers may live on other GPUs (plain peer loads).
+cudaError_t launch_apply_mean_peers(const LaunchPlan& plan, const float* const* buffers, int n_buffers, int n_local,
+                                    double inv_n_global, cudaStream_t stream);
+
 // Diagnostic: a one-CTA kernel whose bounded barrier wait runs out (about a second) and sets bit 1 of *status.
 cudaError_t launch_bounded_wait_probe(unsigned* status, cudaStream_t stream);
 

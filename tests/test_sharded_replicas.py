@@ -81,6 +81,51 @@ class _Rank:
 
 
 @pytest.mark.gpu
+@pytest.mark.parametrize("split", [(2, 2, 2), (3, 1, 2), (6,)])
+def test_exchange_inside_the_kernel_matches_the_oracle_and_agrees_on_every_rank(split):
+    """hdet_apply_mean_peers: every emulated rank reads all staging buffers itself (here all on one device, where a
+    peer's buffer is just another pointer) in rank order; no all-reduce.  Every rank must end with the same bits,
+    and they must be the oracle's mean within the tolerances."""
+    import torch
+    w = W.ragged_workload(n_replicas=6, numels=(4099, 7, 2048, 1, 6150, 33))
+    ranks, off = [], 0
+    for n_local in split:
+        ranks.append(_Rank(w, n_local, off, False))
+        off += n_local
+    o = H.OracleRun(w, H.whole_tensor_slabs(w))
+    stream = torch.cuda.current_stream().cuda_stream
+    for i in range(w.total_steps):
+        perm = list(B.hdet_get_state(ranks[0].h).perm_lr[0])[:6]
+        losses = list(R.step_losses(w, i, perm))
+        ended = None
+        for rk in ranks:
+            rk.fill_grads(i)
+            ended = B.hdet_step_sharded(rk.h, losses, rk.partial, stream)
+        assert ended == o.step()
+        if ended:                                # one stream: the launches below follow every rank's update in order
+            for rk in ranks:
+                B.hdet_apply_mean_peers(rk.h, [q.partial for q in ranks], stream)
+                B.hdet_autolr_update(rk.h)
+            means = [rk.arena.param[0].clone() for rk in ranks]
+            for rk, m in zip(ranks, means):
+                for ao, t in zip(rk.arena.offsets, w.tensors):
+                    assert torch.equal(m[ao:ao + t.numel], means[0][ao:ao + t.numel])          # same bits on every rank
+                    bits = rk.arena.param_bf16[ao:ao + t.numel].view(torch.int16).cpu().numpy().view(np.uint16)
+                    assert np.array_equal(bits, O.bf16_bits(m[ao:ao + t.numel].cpu().numpy()))
+        tol = 1e-6 if i == 0 else 1e-5
+        for rk in ranks:
+            for k, (ao, t) in enumerate(zip(rk.arena.offsets, w.tensors)):
+                got = rk.arena.param[:, ao:ao + t.numel].cpu().numpy()
+                assert H.rel_err(got, o.o.theta[k][rk.offset:rk.offset + rk.n_local]).max() <= tol, (i, k)
+    with pytest.raises(B.HdetError) as e:
+        B.hdet_apply_mean_peers(ranks[0].h, [], stream)
+    assert e.value.status == B.HDET_ERR_INVALID_ARG
+    for rk in ranks:
+        torch.cuda.synchronize()
+        B.hdet_destroy(rk.h)
+
+
+@pytest.mark.gpu
 @pytest.mark.parametrize("shared_grad", [False, True])
 @pytest.mark.parametrize("split", [(2, 2, 2), (3, 1, 2), (6,)])
 def test_sharded_replica_axis_matches_the_oracle_with_all_replicas(split, shared_grad):
