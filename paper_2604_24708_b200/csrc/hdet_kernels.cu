@@ -2,10 +2,14 @@
 //
 // Work assignment: one CTA owns one tile (kTileElems consecutive elements of one tensor)
 // and streams ALL N replicas of that tile, so the replica mean of Eq. 3 is a per-thread
-// register accumulation: no inter-CTA dependence, no atomics on data, no device-side wait.
-// The path is HBM-bound (about 1.5 flop per byte): accesses are 128-bit, warp-contiguous,
-// read-once / write-once with streaming cache hints, and replica r+1 is loaded while
-// replica r is being computed and stored (explicit two-stage register pipeline).
+// register accumulation: no inter-CTA dependence, no atomics on data.
+// The path is HBM-bound (about 1.5 flop per byte).  Two ways of moving a tile:
+//   - AdamW with per-replica moments, full 16-byte-aligned tiles: bulk asynchronous copies into a ring of
+//     shared-memory stages, issued by a producer warp and tracked by shared-memory barriers (tile_bulk);
+//     every wait on a barrier is bounded;
+//   - everything else (SGD, shared moments, ragged or unaligned tiles): 128-bit warp-contiguous accesses,
+//     read-once / write-once with streaming cache hints, replica r+1 loaded while replica r is being
+//     computed and stored (explicit two-stage register pipeline); scalar accesses where alignment demands.
 #include <cuda_bf16.h>
 
 #include <type_traits>
