@@ -358,3 +358,38 @@ def test_work_plan_rejects_what_create_rejects_and_reports_small_capacity():
     cfg = from_workload.config_for(w)
     assert B._lib.hdet_plan_tiles(C.byref(cfg), arr, len(descs), buf, buf, 4, C.byref(count), None, None) == B.HDET_ERR_INVALID_ARG
     assert count.value == sum((t.numel + 2047) // 2048 for t in w.tensors)
+
+
+def test_entry_points_that_need_a_device_say_so_on_a_handle_without_tensors():
+    """A handle without tensors runs only the scalar part: the diagnostic that launches a kernel is refused, the
+    peer-mean has nothing to do, and bad arguments are still reported before any device is touched."""
+    from hdet_inputs import workloads as W
+    from paper_2604_24708_b200 import from_workload
+    w = W.config2()
+    h = B.hdet_create(from_workload.config_for(w, n_local=4, replica_offset=0), [])
+    B.hdet_set_schedule(h, from_workload.schedule_for(w))
+    with pytest.raises(B.HdetError) as e:
+        B.hdet_selftest_bounded_wait(h)
+    assert e.value.status == B.HDET_ERR_UNSUPPORTED
+    B.hdet_apply_mean_peers(h, [0x1000])          # no tiles: nothing to average, no device call
+    assert B.hdet_kernel_launches(h) == 0
+    B.hdet_destroy(h)
+    assert B._lib.hdet_apply_mean_peers(None, None, 0, None) == B.HDET_ERR_INVALID_ARG
+    assert B._lib.hdet_selftest_bounded_wait(None, None) == B.HDET_ERR_INVALID_ARG
+
+
+def test_bf16_copy_pointer_alignment_selects_the_path():
+    from hdet_inputs import workloads as W
+    from paper_2604_24708_b200 import from_workload
+    w = W.ragged_workload(align_elems=8)
+    for misalign, want_big in ((0, 3), (8, 1), (2, 0)):
+        descs = _fake_descriptors(w)
+        for d, off in zip(descs, w.arena_offsets()):
+            d.param_bf16 = 0x7400_0000_0000 + 2 * off + misalign
+        _, _, access, _ = B.hdet_plan_tiles(from_workload.config_for(w), descs)
+        assert set(access) == {want_big}
+    descs = _fake_descriptors(w)
+    descs[0].param_bf16 = 0x7400_0000_0001
+    with pytest.raises(B.HdetError) as e:
+        B.hdet_plan_tiles(from_workload.config_for(w), descs)
+    assert e.value.status == B.HDET_ERR_ALIGN
