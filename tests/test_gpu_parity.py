@@ -412,6 +412,48 @@ def test_bf16_copy_of_the_averaged_parameters(align, mode):
         g.close()
 
 
+@pytest.mark.parametrize("grad_dtype", [W.DTYPE_BF16, W.DTYPE_F32])
+@pytest.mark.parametrize("grad_mean", [False, True])
+def test_bulk_register_and_scalar_paths_give_the_same_bits(grad_dtype, grad_mean):
+    """The same tensors WITH THE SAME VALUES laid out at 8-, 4- and 1-element alignment go through the bulk-copy
+    ring, the 128-bit register pipeline and the scalar path; parameters and both moments must agree bit for bit
+    after a whole run (fused converges included), tensor by tensor.  (The seeded generator indexes by arena
+    offset, so the values of the 8-aligned run are copied into the other layouts tensor by tensor.)"""
+    import torch
+    numels = (6150, 2048, 33, 12289, 4097, 8192)
+    runs = [H.GpuRun(W.ragged_workload(n_replicas=5, grad_dtype=grad_dtype, align_elems=a, numels=numels), grad_mean=grad_mean)
+            for a in (8, 4, 1)]
+    src = runs[0]
+
+    def copy_from_src(name):
+        for g in runs[1:]:
+            for k, ne in enumerate(numels):
+                o0, o1 = src.arena.offsets[k], g.arena.offsets[k]
+                getattr(g.arena, name)[:, o1:o1 + ne].copy_(getattr(src.arena, name)[:, o0:o0 + ne])
+
+    try:
+        copy_from_src("param")
+        w = src.w
+        for i in range(w.total_steps):
+            src.fill_grads(i)
+            copy_from_src("grad")
+            losses = list(R.step_losses(w, i, src.perm0()))
+            for g in runs:
+                if g.B.hdet_step(g.h, losses):
+                    g.B.hdet_autolr_update(g.h)
+        torch.cuda.synchronize()
+        for g in runs[1:]:
+            for k, ne in enumerate(numels):
+                o0, o1 = src.arena.offsets[k], g.arena.offsets[k]
+                for name in ("param", "exp_avg", "exp_avg_sq"):
+                    assert torch.equal(getattr(src.arena, name)[:, o0:o0 + ne], getattr(g.arena, name)[:, o1:o1 + ne]), \
+                        (name, k, g.w.align_elems)
+            assert g.state().device_status == 0
+    finally:
+        for g in runs:
+            g.close()
+
+
 def test_the_first_step_of_a_fresh_handle_can_be_recorded_into_a_cuda_graph():
     """hdet_create prepares the bulk-copy kernels (their shared-memory attribute), so even the very first
     hdet_step of a handle makes no attribute call and can be captured; a replay equals a direct step bit for bit."""
