@@ -234,11 +234,17 @@ HDET_API int hdet_step(hdet_handle h, const double* step_losses, void* stream, i
 /*
  * hdet_step_host_grads -- hdet_step for gradients that live in HOST memory: host_grads[k] points to
  * the gradients of tensor k laid out like its device gradient (replica r at host_grads[k] +
- * r * grad_stride elements; one copy when grad_stride is 0).  The call enqueues the host-to-device
- * copies of all tensors on `stream` (one strided copy per tensor) and then the update, so the copies
- * are inside the call.  The host buffers must stay valid until the stream has passed the copies; they
- * should be pinned, otherwise every copy waits for the stream and stages through the driver.
- * Errors: as hdet_step, plus INVALID_ARG for NULL pointers and CUDA for a failed copy.
+ * r * grad_stride elements; one copy when grad_stride is 0).  The call uploads them into the tensors' device
+ * gradient arrays (one strided copy per tensor) and updates, so the copies are inside the call.  Copies and
+ * updates overlap: the tensor list is cut into up to eight runs of consecutive tensors; the copies go to a
+ * stream the handle creates on its first call here (ordered after everything already enqueued on `stream`),
+ * and `stream` updates each run's tiles as soon as that run's copies have landed -- one kernel launch per run,
+ * same arithmetic and same results as hdet_step on gradients already on the device.  When the call returns
+ * everything is enqueued and later work on `stream` is ordered after all of it.  The host buffers must stay valid
+ * until `stream` has passed the call's work; they should be pinned, otherwise every copy stages through the
+ * driver and blocks.  The first call creates the stream and its events (no device memory).
+ * Errors: as hdet_step, plus INVALID_ARG for NULL pointers and CUDA for a failed copy; nothing is enqueued when
+ * an argument or the handle's state is rejected.
  */
 HDET_API int hdet_step_host_grads(hdet_handle h, const void* const* host_grads, const double* step_losses,
                                   void* stream, int32_t* did_converge);

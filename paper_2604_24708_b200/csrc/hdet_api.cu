@@ -60,6 +60,13 @@ struct hdet_ctx {
   int64_t partial_numel = 0;   // elements of the partial-sum staging buffer
   std::vector<int64_t> partial_offsets;  // per tensor, inside that buffer
   std::vector<hdet_tensor> tensors;      // the caller's descriptors (for hdet_step_host_grads)
+  // hdet_step_host_grads uploads the gradients in a few runs of consecutive tensors on a stream of its own and
+  // updates each run's tiles as soon as its copies have landed, so that copies and updates overlap.
+  struct UploadRun { int64_t first_tensor, n_tensors; int first_tile, n_tiles; };
+  std::vector<UploadRun> upload_runs;
+  cudaStream_t copy_stream = nullptr;    // created by the first hdet_step_host_grads call
+  cudaEvent_t upload_begin = nullptr;
+  std::vector<cudaEvent_t> upload_done;  // one per run
   int64_t launches = 0;
   std::string error;
 };
@@ -100,6 +107,10 @@ void free_device(hdet_ctx* h) {
   if (h->d_status) cudaFree(h->d_status);
   if (h->d_state) cudaFree(h->d_state);
   if (h->d_warm) cudaFree(h->d_warm);
+  if (h->copy_stream) cudaStreamDestroy(h->copy_stream);
+  if (h->upload_begin) cudaEventDestroy(h->upload_begin);
+  for (cudaEvent_t ev : h->upload_done) cudaEventDestroy(ev);
+  h->copy_stream = nullptr; h->upload_begin = nullptr; h->upload_done.clear();
   h->d_warm = nullptr;
   h->d_tensors = nullptr; h->d_tiles = nullptr; h->d_status = nullptr; h->d_state = nullptr;
 }
@@ -345,6 +356,25 @@ int hdet_create(const hdet_config* cfg, const hdet_tensor* tensors, int64_t n_te
   h->r_offset = sharded ? cfg->replica_offset : 0;
   h->partial_numel = partial_numel;
   h->tensors.assign(tensors, tensors + n_tensors);
+  {   // upload runs: at most kUploadRuns runs of consecutive tensors holding about the same number of elements each
+    constexpr int kUploadRuns = 8;
+    const double per_run = h->total_numel / kUploadRuns;
+    hdet_ctx::UploadRun run{0, 0, 0, 0};
+    double in_run = 0.0;
+    int tile_cursor = 0;
+    for (int64_t k = 0; k < n_tensors; ++k) {
+      const int n_tiles_k = (int)((tensors[k].numel + kTileElems - 1) / kTileElems);
+      run.n_tensors += 1;
+      run.n_tiles += n_tiles_k;
+      in_run += (double)tensors[k].numel;
+      tile_cursor += n_tiles_k;
+      if ((in_run >= per_run && (int)h->upload_runs.size() < kUploadRuns - 1) || k == n_tensors - 1) {
+        h->upload_runs.push_back(run);
+        run = hdet_ctx::UploadRun{k + 1, 0, tile_cursor, 0};
+        in_run = 0.0;
+      }
+    }
+  }
   for (const TensorDesc& d : descs) h->partial_offsets.push_back(d.partial_off);
   spread_multipliers(n_global, cfg->alpha_lr, h->rho_lr);
   spread_multipliers(n_global, cfg->alpha_wd, h->rho_wd);
@@ -441,8 +471,28 @@ int hdet_set_schedule(hdet_handle h, const hdet_schedule* s) {
 
 // One loop body of Algorithm 1 with host scalars.  `partial` != NULL: a round's last update writes the
 // sums over the local replicas to `partial` instead of the mean (replica axis sharded over GPUs).
+// Enqueues the host-to-device copies of tensors [first, first + count) on `st` (one strided copy per tensor).
+static cudaError_t upload_gradients(hdet_ctx* h, const void* const* host_grads, int64_t first, int64_t count, cudaStream_t st) {
+  const size_t gsz = h->cfg.grad_dtype == HDET_DTYPE_BF16 ? 2 : 4;
+  for (int64_t k = first; k < first + count; ++k) {
+    const hdet_tensor& t = h->tensors[k];
+    const size_t row = (size_t)t.numel * gsz;
+    cudaError_t e;
+    if (t.grad_stride == 0 || h->cfg.n_replicas == 1) {
+      e = cudaMemcpyAsync(t.grad, host_grads[k], row, cudaMemcpyHostToDevice, st);
+    } else {   // N rows of one tensor, replica stride as pitch on both sides
+      const size_t pitch = (size_t)t.grad_stride * gsz;
+      e = cudaMemcpy2DAsync(t.grad, pitch, host_grads[k], pitch, row, (size_t)h->cfg.n_replicas, cudaMemcpyHostToDevice, st);
+    }
+    if (e != cudaSuccess) return e;
+  }
+  return cudaSuccess;
+}
+
+// `host_grads` != NULL: the gradients are uploaded from host memory first, run by run, each run's tiles updated as
+// soon as its copies have landed (hdet_step_host_grads).
 static int step_impl(hdet_handle h, const double* step_losses, bool sharded_call, float* partial, void* stream,
-                     int32_t* did_converge) {
+                     int32_t* did_converge, const void* const* host_grads = nullptr) {
   if (!h) return HDET_ERR_INVALID_ARG;
   if (did_converge) *did_converge = 0;
   if (!h->has_schedule) return fail(h, HDET_ERR_STATE, "hdet_step: call hdet_set_schedule first");
@@ -483,11 +533,43 @@ static int step_impl(hdet_handle h, const double* step_losses, bool sharded_call
     const bool fuse = ends_round && (h->cfg.fuse_converge || partial);
     LaunchPlan plan{h->d_tensors, h->d_tiles, h->n_tiles, h->grid_fanout, h->d_status, nullptr,
                     ends_round ? partial : nullptr};
-    cudaError_t e = launch_fanout(h->cfg.optimizer, h->cfg.optimizer == HDET_OPT_SGD && h->cfg.momentum != 0.0, h->cfg.grad_dtype, fuse,
-                                  h->cfg.grad_mode == HDET_GRAD_REPLICA_MEAN,
-                                  h->shared_state, plan, s, st);
-    if (e != cudaSuccess) return fail_cuda(h, "hdet_step: fan-out launch", e);
-    ++h->launches;
+    const bool sgd_momentum = h->cfg.optimizer == HDET_OPT_SGD && h->cfg.momentum != 0.0;
+    const bool grad_mean = h->cfg.grad_mode == HDET_GRAD_REPLICA_MEAN;
+    cudaError_t e = cudaSuccess;
+    if (!host_grads) {
+      e = launch_fanout(h->cfg.optimizer, sgd_momentum, h->cfg.grad_dtype, fuse, grad_mean, h->shared_state, plan, s, st);
+      if (e != cudaSuccess) return fail_cuda(h, "hdet_step: fan-out launch", e);
+      ++h->launches;
+    } else {
+      // Copies run on the handle's own stream, ordered after everything already enqueued on the caller's stream;
+      // the caller's stream waits for each run's copies and then updates that run's tiles.
+      if (!h->copy_stream) {
+        e = cudaStreamCreateWithFlags(&h->copy_stream, cudaStreamNonBlocking);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->upload_begin, cudaEventDisableTiming);
+        for (size_t c = 0; e == cudaSuccess && c < h->upload_runs.size(); ++c) {
+          cudaEvent_t ev = nullptr;
+          e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming);
+          if (e == cudaSuccess) h->upload_done.push_back(ev);
+        }
+        if (e != cudaSuccess) return fail_cuda(h, "hdet_step_host_grads: stream and events", e);
+      }
+      e = cudaEventRecord(h->upload_begin, st);
+      if (e == cudaSuccess) e = cudaStreamWaitEvent(h->copy_stream, h->upload_begin, 0);
+      for (size_t c = 0; e == cudaSuccess && c < h->upload_runs.size(); ++c) {
+        const hdet_ctx::UploadRun& run = h->upload_runs[c];
+        e = upload_gradients(h, host_grads, run.first_tensor, run.n_tensors, h->copy_stream);
+        if (e == cudaSuccess) e = cudaEventRecord(h->upload_done[c], h->copy_stream);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(st, h->upload_done[c], 0);
+        if (e != cudaSuccess) break;
+        LaunchPlan part = plan;
+        part.tiles = h->d_tiles + run.first_tile;
+        part.n_tiles = run.n_tiles;
+        part.grid = run.n_tiles;
+        e = launch_fanout(h->cfg.optimizer, sgd_momentum, h->cfg.grad_dtype, fuse, grad_mean, h->shared_state, part, s, st);
+        if (e == cudaSuccess) ++h->launches;
+      }
+      if (e != cudaSuccess) return fail_cuda(h, "hdet_step_host_grads: upload and update", e);
+    }
     if (ends_round && !fuse) {
       plan.grid = h->grid_converge;
       e = launch_converge(plan, n, st);
@@ -524,27 +606,9 @@ int hdet_step_host_grads(hdet_handle h, const void* const* host_grads, const dou
   if (!h) return HDET_ERR_INVALID_ARG;
   if (did_converge) *did_converge = 0;
   if (h->n_tensors > 0 && !host_grads) return fail(h, HDET_ERR_INVALID_ARG, "hdet_step_host_grads: host_grads is NULL");
-  if (h->n_tensors > 0) {
-    DeviceScope scope(h->cfg.device);
-    if (scope.err != cudaSuccess) return fail_cuda(h, "hdet_step_host_grads", scope.err);
-    const size_t gsz = h->cfg.grad_dtype == HDET_DTYPE_BF16 ? 2 : 4;
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    for (int64_t k = 0; k < h->n_tensors; ++k) {
-      const hdet_tensor& t = h->tensors[k];
-      if (!host_grads[k]) return fail(h, HDET_ERR_INVALID_ARG, "hdet_step_host_grads: a host gradient pointer is NULL");
-      const size_t row = (size_t)t.numel * gsz;
-      cudaError_t e;
-      if (t.grad_stride == 0 || h->cfg.n_replicas == 1) {
-        e = cudaMemcpyAsync(t.grad, host_grads[k], row, cudaMemcpyHostToDevice, st);
-      } else {   // N rows of one tensor, replica stride as pitch on both sides
-        const size_t pitch = (size_t)t.grad_stride * gsz;
-        e = cudaMemcpy2DAsync(t.grad, pitch, host_grads[k], pitch, row, (size_t)h->cfg.n_replicas,
-                              cudaMemcpyHostToDevice, st);
-      }
-      if (e != cudaSuccess) return fail_cuda(h, "hdet_step_host_grads: gradient upload", e);
-    }
-  }
-  return step_impl(h, step_losses, false, nullptr, stream, did_converge);
+  for (int64_t k = 0; k < h->n_tensors; ++k)
+    if (!host_grads[k]) return fail(h, HDET_ERR_INVALID_ARG, "hdet_step_host_grads: a host gradient pointer is NULL");
+  return step_impl(h, step_losses, false, nullptr, stream, did_converge, h->n_tensors > 0 ? host_grads : nullptr);
 }
 
 int hdet_step_sharded(hdet_handle h, const double* step_losses, void* d_partial, void* stream, int32_t* did_converge) {
@@ -828,7 +892,7 @@ int hdet_selftest_bounded_wait(hdet_handle h, void* stream) {
 int hdet_destroy(hdet_handle h) {
   TraceRange trace("hdet_destroy");
   if (!h) return HDET_OK;
-  if (h->d_tensors || h->d_tiles || h->d_status || h->d_state || h->d_warm) {
+  if (h->d_tensors || h->d_tiles || h->d_status || h->d_state || h->d_warm || h->copy_stream) {
     DeviceScope scope(h->cfg.device);
     free_device(h);
   }
