@@ -591,7 +591,7 @@ template <int kOpt>
 constexpr bool kHasBulkPath = kOpt == kOptAdamW;
 
 template <typename GradT, int kOpt, bool kConv, bool kMean>
-__global__ void __launch_bounds__(kHasBulkPath<kOpt> ? kThreads + kProducerThreads : kThreads, 2)
+__global__ void __launch_bounds__(kHasBulkPath<kOpt> ? kThreads + kProducerThreads : kThreads, (kOpt == kOptSgd && !kMean) ? 3 : 2)
 fanout_kernel(const __grid_constant__ LaunchPlan plan, const __grid_constant__ StepScalars s_param) {
   __shared__ StepScalars s;
   if constexpr (kHasBulkPath<kOpt>) {
